@@ -1,0 +1,387 @@
+// C ABI of the library: argument checking, TMA tensor-map encoding and kernel launches.
+// Everything here runs on the host; no device memory is allocated and nothing synchronises
+// except pevlm_read_status.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "internal.h"
+
+namespace pevlm {
+
+static thread_local char g_cuda_error[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+    return PEVLM_ECUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+static int check_shape(const pevlm_shape_t* s) {
+    if (!s) return PEVLM_EINVAL;
+    if (s->batch < 1 || s->sink_len < 0 || s->num_blocks < 0 || s->query_len < 0) return PEVLM_EINVAL;
+    if (s->num_blocks > 0 && s->block_len < 1) return PEVLM_EINVAL;
+    if (s->block_len < 0) return PEVLM_EINVAL;
+    if (s->num_q_heads < 1 || s->num_kv_heads < 1 || s->num_q_heads % s->num_kv_heads != 0) return PEVLM_EINVAL;
+    if (s->mask_mode != PEVLM_MASK_PEVLM && s->mask_mode != PEVLM_MASK_FULL_CAUSAL) return PEVLM_EINVAL;
+    if (!(s->rope_theta > 0.f) || !(s->softmax_scale >= 0.f)) return PEVLM_EINVAL;
+    const int64_t L = static_cast<int64_t>(s->sink_len) + static_cast<int64_t>(s->num_blocks) * s->block_len + s->query_len;
+    if (L < 1 || L > (1ll << 30)) return PEVLM_EINVAL;
+    if (s->head_dim != 64 && s->head_dim != 128) return PEVLM_EUNSUPPORTED;
+    if (s->num_q_heads / s->num_kv_heads > kTile) return PEVLM_EUNSUPPORTED;
+    return PEVLM_OK;
+}
+
+static int64_t n_video(const pevlm_shape_t* s) {
+    return static_cast<int64_t>(s->sink_len) + static_cast<int64_t>(s->num_blocks) * s->block_len;
+}
+
+static int check_device() {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    if (major != 10) return PEVLM_EUNSUPPORTED;
+    return PEVLM_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map over a [tokens, heads, d] bf16 tensor (d contiguous) with a box of
+// 64 elements x box_heads x box_tokens and the 128-byte swizzle the MMA descriptors expect.
+// Rows past the end of the tensor read as zero.
+static int make_tmap(CUtensorMap* m, const void* base, int64_t tokens, int heads, int d, int box_heads, int box_tokens) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled entry point not found");
+        return PEVLM_ECUDA;
+    }
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(tokens)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(d) * 2 * heads};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_heads), static_cast<cuuint32_t>(box_tokens)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+        return PEVLM_ECUDA;
+    }
+    return PEVLM_OK;
+}
+
+static float resolve_scale(const pevlm_shape_t* s) {
+    return s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf(static_cast<float>(s->head_dim));
+}
+
+// ---- question-attention decomposition (shared by the launch, the workspace size and the stats)
+struct QueryPlan {
+    int tok_per_tile, q_tiles, total_kv_tiles, n_splits, tiles_per_split;
+};
+
+static QueryPlan plan_query(const pevlm_shape_t* s) {
+    QueryPlan q;
+    const int G = s->num_q_heads / s->num_kv_heads;
+    const int64_t L = n_video(s) + s->query_len;
+    q.tok_per_tile = kTile / G;
+    q.q_tiles = (s->query_len + q.tok_per_tile - 1) / q.tok_per_tile;
+    q.total_kv_tiles = static_cast<int>((L + kTile - 1) / kTile);
+    const int groups = s->num_kv_heads * (q.q_tiles > 0 ? q.q_tiles : 1);
+    int want = (2 * 148 + groups - 1) / groups;  // about two CTAs per SM
+    if (want < 1) want = 1;
+    if (want > q.total_kv_tiles) want = q.total_kv_tiles;
+    q.tiles_per_split = (q.total_kv_tiles + want - 1) / want;
+    q.n_splits = (q.total_kv_tiles + q.tiles_per_split - 1) / q.tiles_per_split;
+    return q;
+}
+
+static size_t query_partial_floats(const pevlm_shape_t* s, const QueryPlan& q) {
+    return static_cast<size_t>(q.n_splits) * s->query_len * s->num_q_heads * (s->head_dim + 1);
+}
+
+}  // namespace pevlm
+
+using namespace pevlm;
+
+extern "C" {
+
+const char* pevlm_strerror(int code) {
+    switch (code) {
+        case PEVLM_OK: return "ok";
+        case PEVLM_EINVAL: return "invalid shape or NULL pointer";
+        case PEVLM_EALIGN: return "pointer not 16-byte aligned (workspace: 256-byte)";
+        case PEVLM_EUNSUPPORTED: return "unsupported head_dim / group size, or device is not sm_100";
+        case PEVLM_EWORKSPACE: return "workspace missing or too small";
+        case PEVLM_ECUDA: return "CUDA error (see pevlm_last_cuda_error)";
+        case PEVLM_ETIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown pevlm status";
+    }
+}
+
+const char* pevlm_last_cuda_error(void) { return g_cuda_error; }
+
+size_t pevlm_workspace_bytes(const pevlm_shape_t* s, int which) {
+    if (check_shape(s) != PEVLM_OK) return 0;
+    if (which == PEVLM_WS_PREFILL) return kStatusBytes;
+    if (which == PEVLM_WS_QUERY) {
+        const QueryPlan q = plan_query(s);
+        return kStatusBytes + static_cast<size_t>(s->batch) * ((query_partial_floats(s, q) * sizeof(float) + 255) / 256 * 256);
+    }
+    return 0;
+}
+
+int pevlm_rope_qk(const pevlm_shape_t* s, const void* q_in, const void* k_in, void* q_out, void* k_out,
+                  int64_t first_token, int64_t n_tokens, const int32_t* pos_ids, void* stream) {
+    int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if (n_tokens < 0 || first_token < 0 || first_token + n_tokens > (1ll << 31)) return PEVLM_EINVAL;
+    if ((q_in == nullptr) != (q_out == nullptr) || (k_in == nullptr) != (k_out == nullptr)) return PEVLM_EINVAL;
+    if (!q_in && !k_in) return PEVLM_EINVAL;
+    if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(q_out) || !aligned16(k_out)) return PEVLM_EALIGN;
+    if (pos_ids && (reinterpret_cast<uintptr_t>(pos_ids) & 3u)) return PEVLM_EALIGN;
+    if (n_tokens == 0) return PEVLM_OK;
+    RopeParams p;
+    const int d = s->head_dim;
+    for (int i = 0; i < d / 2; ++i) p.inv_freq[i] = pow(static_cast<double>(s->rope_theta), -2.0 * i / d);
+    for (int i = d / 2; i < 64; ++i) p.inv_freq[i] = 0.0;
+    p.first_token = first_token;
+    p.n_tokens = n_tokens;
+    p.Hq = q_in ? s->num_q_heads : 0;
+    p.Hkv = k_in ? s->num_kv_heads : 0;
+    for (int b = 0; b < s->batch; ++b) {
+        const int64_t qo = static_cast<int64_t>(b) * n_tokens * s->num_q_heads * d;
+        const int64_t ko = static_cast<int64_t>(b) * n_tokens * s->num_kv_heads * d;
+        p.q_in = q_in ? static_cast<const __nv_bfloat16*>(q_in) + qo : nullptr;
+        p.q_out = q_out ? static_cast<__nv_bfloat16*>(q_out) + qo : nullptr;
+        p.k_in = k_in ? static_cast<const __nv_bfloat16*>(k_in) + ko : nullptr;
+        p.k_out = k_out ? static_cast<__nv_bfloat16*>(k_out) + ko : nullptr;
+        p.pos_ids = pos_ids ? pos_ids + static_cast<int64_t>(b) * n_tokens : nullptr;
+        cudaError_t e = launch_rope(p, d, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "rope launch");
+    }
+    return PEVLM_OK;
+}
+
+int pevlm_assemble_kv(const pevlm_shape_t* s, const void* k_video, const void* v_video, const void* k_question,
+                      const void* v_question, void* k_cache, void* v_cache, void* stream) {
+    int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if ((k_video || k_question) && !k_cache) return PEVLM_EINVAL;
+    if ((v_video || v_question) && !v_cache) return PEVLM_EINVAL;
+    if (!aligned16(k_video) || !aligned16(v_video) || !aligned16(k_question) || !aligned16(v_question) ||
+        !aligned16(k_cache) || !aligned16(v_cache))
+        return PEVLM_EALIGN;
+    const int64_t nv = n_video(s);
+    const int64_t row_vec = static_cast<int64_t>(s->num_kv_heads) * s->head_dim * 2 / 16;  // 16-byte vectors per token
+    const int64_t L = nv + s->query_len;
+    for (int b = 0; b < s->batch; ++b) {
+        CopySegments seg;
+        const void* srcs[4] = {k_video, k_question, v_video, v_question};
+        void* dsts[4] = {k_cache, k_cache, v_cache, v_cache};
+        const int64_t rows[4] = {nv, s->query_len, nv, s->query_len};
+        const int64_t dst_row0[4] = {0, nv, 0, nv};
+        seg.total = 0;
+        for (int i = 0; i < 4; ++i) {
+            const int64_t n = srcs[i] ? rows[i] * row_vec : 0;
+            seg.n_vec[i] = n;
+            seg.src[i] = srcs[i] ? static_cast<const uint4*>(srcs[i]) + static_cast<int64_t>(b) * rows[i] * row_vec : nullptr;
+            seg.dst[i] = dsts[i] ? static_cast<uint4*>(dsts[i]) + (static_cast<int64_t>(b) * L + dst_row0[i]) * row_vec : nullptr;
+            seg.total += n;
+        }
+        cudaError_t e = launch_copy_segments(seg, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "assemble launch");
+    }
+    return PEVLM_OK;
+}
+
+int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const void* k, const void* v, void* o, float* lse,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if (!q || !k || !v || !o) return PEVLM_EINVAL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return PEVLM_EALIGN;
+    if (!workspace || workspace_bytes < pevlm_workspace_bytes(s, PEVLM_WS_PREFILL)) return PEVLM_EWORKSPACE;
+    if (!aligned256(workspace)) return PEVLM_EALIGN;
+    const int64_t nv = n_video(s);
+    if (nv == 0) return PEVLM_OK;
+    rc = check_device();
+    if (rc != PEVLM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
+
+    const int d = s->head_dim;
+    AttnParams p;
+    memset(&p, 0, sizeof(p));
+    p.mode = 0;
+    if (s->mask_mode == PEVLM_MASK_FULL_CAUSAL) {
+        p.S = 0; p.B = static_cast<int>(nv); p.N = 1;
+    } else {
+        p.S = s->sink_len; p.B = s->num_blocks > 0 ? s->block_len : 0; p.N = s->num_blocks;
+    }
+    p.n_video = static_cast<int>(nv);
+    p.Q = s->query_len;
+    p.L = static_cast<int>(nv + s->query_len);
+    p.Hq = s->num_q_heads; p.Hkv = s->num_kv_heads; p.G = p.Hq / p.Hkv;
+    p.tiles_sink = (p.S + kTile - 1) / kTile;
+    p.tiles_block = p.N > 0 ? (p.B + kTile - 1) / kTile : 0;
+    p.items_block = p.N * p.tiles_block * p.Hq;
+    p.n_items = p.items_block + p.tiles_sink * p.Hq;
+    p.q_box_rows = kTile;
+    p.scale = resolve_scale(s);
+    p.scale_log2 = p.scale * 1.4426950408889634f;
+    p.hdr = static_cast<WorkspaceHeader*>(workspace);
+    for (int b = 0; b < s->batch; ++b) {
+        const int64_t qoff = static_cast<int64_t>(b) * nv * p.Hq * d, koff = static_cast<int64_t>(b) * nv * p.Hkv * d;
+        CUtensorMap tq, tk, tv;
+        if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q) + qoff, nv, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        p.o = static_cast<__nv_bfloat16*>(o) + qoff;
+        p.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * nv : nullptr;
+        e = launch_attn(p, d, tq, tk, tv, st);
+        if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
+    }
+    return PEVLM_OK;
+}
+
+int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void* k_cache, const void* v_cache, void* o,
+                     float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if (!q_question || !k_cache || !v_cache || !o) return PEVLM_EINVAL;
+    if (!aligned16(q_question) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(lse))
+        return PEVLM_EALIGN;
+    if (!workspace || workspace_bytes < pevlm_workspace_bytes(s, PEVLM_WS_QUERY)) return PEVLM_EWORKSPACE;
+    if (!aligned256(workspace)) return PEVLM_EALIGN;
+    if (s->query_len == 0) return PEVLM_OK;
+    rc = check_device();
+    if (rc != PEVLM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
+
+    const int d = s->head_dim;
+    const int64_t nv = n_video(s);
+    const int64_t L = nv + s->query_len;
+    const QueryPlan qp = plan_query(s);
+    AttnParams p;
+    memset(&p, 0, sizeof(p));
+    p.mode = 1;
+    p.n_video = static_cast<int>(nv);
+    p.Q = s->query_len;
+    p.L = static_cast<int>(L);
+    p.Hq = s->num_q_heads; p.Hkv = s->num_kv_heads; p.G = p.Hq / p.Hkv;
+    p.tok_per_tile = qp.tok_per_tile;
+    p.q_tiles = qp.q_tiles;
+    p.n_splits = qp.n_splits;
+    p.tiles_per_split = qp.tiles_per_split;
+    p.q_box_rows = p.G * p.tok_per_tile;
+    p.n_items = p.Hkv * p.q_tiles * p.n_splits;
+    p.scale = resolve_scale(s);
+    p.scale_log2 = p.scale * 1.4426950408889634f;
+    p.hdr = static_cast<WorkspaceHeader*>(workspace);
+    const size_t part_floats = query_partial_floats(s, qp);
+    const size_t part_stride = (part_floats * sizeof(float) + 255) / 256 * 256;
+    for (int b = 0; b < s->batch; ++b) {
+        float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes + b * part_stride);
+        p.part_o = part;
+        p.part_lse = part + static_cast<size_t>(p.n_splits) * p.Q * p.Hq * d;
+        const int64_t qoff = static_cast<int64_t>(b) * p.Q * p.Hq * d, koff = static_cast<int64_t>(b) * L * p.Hkv * d;
+        CUtensorMap tq, tk, tv;
+        if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        e = launch_attn(p, d, tq, tk, tv, st);
+        if (e != cudaSuccess) return cuda_fail(e, "question attention launch");
+        MergeParams m;
+        m.Q = p.Q; m.Hq = p.Hq; m.d = d; m.n_splits = p.n_splits;
+        m.part_o = p.part_o; m.part_lse = p.part_lse;
+        m.o = static_cast<__nv_bfloat16*>(o) + qoff;
+        m.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * p.Q : nullptr;
+        e = launch_merge(m, st);
+        if (e != cudaSuccess) return cuda_fail(e, "merge launch");
+    }
+    return PEVLM_OK;
+}
+
+int pevlm_read_status(const void* workspace, void* stream, int32_t* status, int32_t* detail) {
+    if (!workspace || !status) return PEVLM_EINVAL;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    int32_t words[2] = {0, 0};
+    e = cudaMemcpy(words, workspace, sizeof(words), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    *status = words[0];
+    if (detail) *detail = words[1];
+    return PEVLM_OK;
+}
+
+int pevlm_tile_stats(const pevlm_shape_t* s, int which, int64_t* tiles, double* flops) {
+    int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if (!tiles || !flops) return PEVLM_EINVAL;
+    const int d = s->head_dim;
+    int64_t n_tiles = 0;
+    double cols = 0.0;  // sum over visited tiles of issued key columns (each over 128 query rows)
+    auto add_range = [&](int64_t len) {  // a key range visited from its start in 128-key tiles
+        for (int64_t j = 0; j < len; j += kTile) {
+            const int64_t valid = len - j < kTile ? len - j : kTile;
+            n_tiles += 1;
+            cols += static_cast<double>((valid + 15) / 16 * 16);
+        }
+    };
+    const int64_t nv = n_video(s);
+    if (which == PEVLM_WS_PREFILL) {
+        int64_t S = s->sink_len, B = s->num_blocks > 0 ? s->block_len : 0, N = s->num_blocks;
+        if (s->mask_mode == PEVLM_MASK_FULL_CAUSAL) { S = 0; B = nv; N = nv > 0 ? 1 : 0; }
+        for (int64_t q0 = 0; q0 < S; q0 += kTile) add_range((q0 + kTile < S ? q0 + kTile : S));
+        const int64_t t0 = n_tiles; const double c0 = cols;
+        for (int64_t q0 = 0; q0 < B; q0 += kTile) { add_range(S); add_range((q0 + kTile < B ? q0 + kTile : B)); }
+        // the block part repeats for each of the N blocks
+        n_tiles = t0 + (n_tiles - t0) * N;
+        cols = c0 + (cols - c0) * static_cast<double>(N);
+        n_tiles *= s->num_q_heads;
+        cols *= s->num_q_heads;
+    } else if (which == PEVLM_WS_QUERY) {
+        const QueryPlan qp = plan_query(s);
+        for (int qt = 0; qt < qp.q_tiles; ++qt) {
+            const int tok0 = qt * qp.tok_per_tile;
+            const int ntok = s->query_len - tok0 < qp.tok_per_tile ? s->query_len - tok0 : qp.tok_per_tile;
+            const int64_t kv_end = nv + tok0 + ntok;
+            for (int sp = 0; sp < qp.n_splits; ++sp) {
+                int64_t a = static_cast<int64_t>(sp) * qp.tiles_per_split * kTile, e = a + static_cast<int64_t>(qp.tiles_per_split) * kTile;
+                if (a > kv_end) a = kv_end;
+                if (e > kv_end) e = kv_end;
+                add_range(e - a);
+            }
+        }
+        n_tiles *= s->num_kv_heads;
+        cols *= s->num_kv_heads;
+    } else {
+        return PEVLM_EINVAL;
+    }
+    *tiles = n_tiles * s->batch;
+    *flops = 4.0 * d * kTile * cols * s->batch;
+    return PEVLM_OK;
+}
+
+}  // extern "C"

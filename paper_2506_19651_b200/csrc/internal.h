@@ -1,0 +1,83 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/pevlm.h"
+
+namespace pevlm {
+
+constexpr int kTile = 128;        // query-tile rows (MMA M) and key-tile columns (MMA N max)
+constexpr int kStatusBytes = 256; // first bytes of every workspace: status word + detail + counters
+
+// Workspace header (device memory, first kStatusBytes of the workspace).
+struct WorkspaceHeader {
+    int32_t status;  // 0 or PEVLM_ETIMEOUT
+    int32_t detail;  // which wait expired (kernel-specific code)
+    int32_t work_counter;
+    int32_t pad[61];
+};
+
+// What one launch of the attention kernel does.  mode 0: prefill rows (sink + blocks, or
+// full causal); mode 1: question rows against the assembled cache, split over keys.
+struct AttnParams {
+    int32_t mode;
+    int32_t S, B, N;        // prefill geometry (full causal: S = 0, B = n_video, N = 1)
+    int32_t n_video;        // S + N*B
+    int32_t Q, L;           // question length, total length
+    int32_t Hq, Hkv, G;
+    int32_t tiles_sink;     // ceil(S / 128)
+    int32_t tiles_block;    // ceil(B / 128)
+    int32_t items_block;    // N * tiles_block * Hq
+    int32_t n_items;        // grid size
+    int32_t q_box_rows;     // rows the Q TMA box brings in (128 prefill, G * tok_per_tile question)
+    int32_t tok_per_tile;   // mode 1: question tokens per query tile = 128 / G
+    int32_t q_tiles;        // mode 1: ceil(Q / tok_per_tile)
+    int32_t n_splits;       // mode 1
+    int32_t tiles_per_split;// mode 1
+    float scale;            // softmax scale
+    float scale_log2;       // scale * log2(e)
+    __nv_bfloat16* o;       // mode 0: [n_video, Hq, d]
+    float* lse;             // mode 0: [Hq, n_video] or NULL
+    float* part_o;          // mode 1: [n_splits, Q, Hq, d] fp32
+    float* part_lse;        // mode 1: [n_splits, Q, Hq]
+    WorkspaceHeader* hdr;
+};
+
+struct MergeParams {
+    int32_t Q, Hq, d, n_splits;
+    const float* part_o;
+    const float* part_lse;
+    __nv_bfloat16* o;  // [Q, Hq, d]
+    float* lse;        // [Hq, Q] or NULL
+};
+
+struct RopeParams {
+    double inv_freq[64];  // theta^(-2i/d), i < d/2, computed on the host in fp64
+    const __nv_bfloat16* q_in;
+    const __nv_bfloat16* k_in;
+    __nv_bfloat16* q_out;
+    __nv_bfloat16* k_out;
+    const int32_t* pos_ids;
+    int64_t first_token;
+    int64_t n_tokens;
+    int32_t Hq, Hkv;  // heads to process of each tensor (0 = skip tensor)
+};
+
+struct CopySegments {
+    const uint4* src[4];
+    uint4* dst[4];
+    int64_t n_vec[4];  // 16-byte vectors per segment
+    int64_t total;
+};
+
+cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream);
+cudaError_t launch_copy_segments(const CopySegments& s, cudaStream_t stream);
+cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
+                        const CUtensorMap& tv, cudaStream_t stream);
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+size_t attn_smem_bytes(int head_dim);
+
+}  // namespace pevlm

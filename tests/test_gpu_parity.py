@@ -1,0 +1,148 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the
+same seeded inputs.  Tolerances: 2e-2 max-abs on outputs, 1e-3 on per-row LSE; RoPE and the
+KV assembly are compared bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import api as oracle
+from paper_2506_19651_b200 import inputs
+from helpers import (LSE_TOL, O_TOL, bits_to_f64, check_against_oracle, gpu_shape, run_gpu_layer, to_bits, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+def wl(S, B, N, Q, Hq, Hkv, d, theta=1e6, outliers=False, seed=1234):
+    return inputs.Workload("t", S, B, N, Q, Hq, Hkv, d, theta, outliers, seed)
+
+
+# ---------------------------------------------------------------- RoPE (Sec. 3.2.2)
+
+@pytest.mark.parametrize("n,Hq,Hkv,d,theta,first", [
+    (37, 4, 2, 64, 1e4, 0), (130, 28, 4, 128, 1e6, 0), (65, 8, 8, 128, 1e6, 70000), (5, 2, 1, 64, 1e6, 123456)])
+def test_rope_bit_exact(n, Hq, Hkv, d, theta, first):
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(n, 1, 0, 0, Hq, Hkv, d, theta)
+    q, k, _ = inputs.make_qkv(w)
+    s = gpu_shape(w)
+    qd, kd = to_dev(q), to_dev(k)
+    qo, ko = torch.empty_like(qd), torch.empty_like(kd)
+    pb.pevlm_rope_qk(s, qd, kd, qo, ko, first, n)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_bits(qo), oracle.rope(q, theta, first_pos=first))
+    np.testing.assert_array_equal(to_bits(ko), oracle.rope(k, theta, first_pos=first))
+    # in place, K only, explicit position ids
+    pos = np.random.default_rng(0).integers(0, 80000, size=n).astype(np.int32)
+    pb.pevlm_rope_qk(s, None, kd, None, kd, 0, n, torch.from_numpy(pos).cuda())
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_bits(kd), oracle.rope(k, theta, pos=pos.astype(np.int64)))
+    np.testing.assert_array_equal(to_bits(qd), q)  # untouched
+
+
+# ---------------------------------------------------------------- KV assembly (Eq. 5 key set)
+
+def test_assemble_kv_bit_exact():
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(100, 77, 3, 19, 4, 2, 64)
+    _, k, v = inputs.make_qkv(w)
+    nv = w.n_video
+    s = gpu_shape(w)
+    kc = torch.zeros((w.L, w.Hkv, w.d), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    pb.pevlm_assemble_kv(s, to_dev(k[:nv]), to_dev(v[:nv]), to_dev(k[nv:]), to_dev(v[nv:]), kc, vc)
+    torch.cuda.synchronize()
+    sh = oracle.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d)
+    np.testing.assert_array_equal(to_bits(kc), oracle.assemble_kv(sh, k[:nv], k[nv:]))
+    np.testing.assert_array_equal(to_bits(vc), oracle.assemble_kv(sh, v[:nv], v[nv:]))
+    # partial call: only the question V rows
+    vc.zero_()
+    pb.pevlm_assemble_kv(s, None, None, None, to_dev(v[nv:]), kc, vc)
+    torch.cuda.synchronize()
+    got = to_bits(vc)
+    np.testing.assert_array_equal(got[nv:], v[nv:])
+    assert (got[:nv] == 0).all()
+
+
+# ---------------------------------------------------------------- whole path, small shapes
+
+SMALL = [
+    # S, B, N, Q, Hq, Hkv, d, theta, outliers
+    (64, 128, 4, 32, 4, 2, 64, 1e4, False),      # the tiny correctness configuration
+    (200, 300, 3, 20, 4, 2, 128, 1e6, True),     # several tiles, ragged tails, outlier sink keys
+    (16, 16, 5, 3, 2, 1, 128, 1e6, False),       # everything smaller than a tile
+    (0, 150, 2, 9, 7, 1, 128, 1e6, False),       # no sink (block attention without sink), G = 7
+    (129, 1, 3, 1, 2, 2, 64, 1e4, False),        # blocks of one token
+    (257, 384, 2, 130, 8, 2, 128, 1e6, True),    # question longer than a tile's worth of tokens
+    (130, 0, 0, 0, 4, 4, 128, 1e6, False),       # sink only
+    (0, 0, 0, 40, 4, 2, 64, 1e4, False),         # question only
+]
+
+
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d,theta,outl", SMALL)
+def test_layer_matches_oracle_small(S, B, N, Q, Hq, Hkv, d, theta, outl):
+    w = wl(S, B, N, Q, Hq, Hkv, d, theta, outl)
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v)
+    errs, qr, kr = check_against_oracle(w, q, k, v, res, np.arange(w.L))
+    nv = w.n_video
+    # RoPE outputs and the assembled cache, bit for bit
+    np.testing.assert_array_equal(res["q_video"], qr[:nv])
+    np.testing.assert_array_equal(res["q_question"], qr[nv:])
+    np.testing.assert_array_equal(res["k_cache"], kr)
+    np.testing.assert_array_equal(res["v_cache"], v)
+    for name, e in errs.items():
+        assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)
+
+
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d", [(100, 200, 2, 10, 4, 2, 128), (64, 128, 4, 32, 4, 2, 64)])
+def test_full_causal_mode_matches_oracle(S, B, N, Q, Hq, Hkv, d):
+    w = wl(S, B, N, Q, Hq, Hkv, d)
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v, full_causal=True)
+    errs, _, _ = check_against_oracle(w, q, k, v, res, np.arange(w.L), full_causal=True)
+    for name, e in errs.items():
+        assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)
+
+
+def test_run_twice_is_bit_identical():
+    w = wl(200, 300, 3, 20, 4, 2, 128, outliers=True)
+    q, k, v = inputs.make_qkv(w)
+    a = run_gpu_layer(w, q, k, v)
+    b = run_gpu_layer(w, q, k, v)
+    for name in ("o_video", "lse_video", "o_question", "lse_question"):
+        np.testing.assert_array_equal(a[name], b[name])
+
+
+def test_softmax_scale_and_null_lse():
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(70, 90, 2, 0, 2, 1, 64, 1e4)
+    q, k, v = inputs.make_qkv(w)
+    qr, kr = oracle.rope(q, w.theta), oracle.rope(k, w.theta)
+    s = gpu_shape(w, scale=0.3)
+    o = torch.empty((w.L, w.Hq, w.d), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device="cuda")
+    pb.pevlm_parallel_prefill_attn(s, to_dev(qr), to_dev(kr), to_dev(v), o, None, ws)
+    torch.cuda.synchronize()
+    ref, _ = oracle.attn_rows(oracle.make_shape(w.S, w.B, w.N, 0, w.Hq, w.Hkv, w.d), qr, kr, v, np.arange(w.L), scale=0.3)
+    assert np.abs(bits_to_f64(to_bits(o)) - ref).max() <= O_TOL
+
+
+# ---------------------------------------------------------------- full-size workloads, sampled rows
+
+@pytest.mark.parametrize("name,n_random", [("c2_qwen", 300), ("c3_long", 150)])
+def test_full_size_sampled_rows(name, n_random):
+    w = inputs.WORKLOADS[name]
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v)
+    rows = inputs.sample_rows(w, n_random)
+    errs, qr, kr = check_against_oracle(w, q, k, v, res, rows)
+    mism_q = int((res["q_video"] != qr[:w.n_video]).sum())
+    mism_k = int((res["k_cache"] != kr).sum())
+    # fp64 sin/cos of the device and of the host libm may differ in the last place; after the
+    # rounding to bf16 that can flip about one element in 1e8 by one bf16 ulp
+    assert mism_q <= 4 and mism_k <= 2, (mism_q, mism_k)
+    np.testing.assert_array_equal(res["v_cache"], v)
+    for key, e in errs.items():
+        assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)

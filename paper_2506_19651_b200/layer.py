@@ -27,8 +27,8 @@ class LayerBuffers:
         self.lse_video = torch.empty((Hq, max(nv, 1)), dtype=f32, device=device)
         self.o_question = torch.empty((max(Q, 1), Hq, d), dtype=bf, device=device)
         self.lse_question = torch.empty((Hq, max(Q, 1)), dtype=f32, device=device)
-        self.ws_prefill = torch.empty(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device=device)
-        self.ws_query = torch.empty(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device=device)
+        self.ws_prefill = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device=device)
+        self.ws_query = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device=device)
 
 
 def layer_forward(buf: LayerBuffers, q, k, v):

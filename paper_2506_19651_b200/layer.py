@@ -31,20 +31,32 @@ class LayerBuffers:
         self.ws_query = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device=device)
 
 
-def layer_forward(buf: LayerBuffers, q, k, v):
+KERNELS_PER_PASS = 7  # rope, V copy, prefill attention, rope, V copy, question attention, merge
+
+
+def layer_forward(buf: LayerBuffers, q, k, v, mark=None):
     """q [L,Hq,d], k, v [L,Hkv,d]: un-roped bf16 device tensors of the whole stream.
-    Leaves O/LSE of the video rows and of the question rows in `buf`."""
+    Leaves O/LSE of the video rows and of the question rows in `buf`.  `mark(name)`, if
+    given, is called before the first call and after each C-ABI call (for event timing)."""
     s = buf.shape
     nv, Q = s.n_video, s.query_len
+    mark = mark or (lambda name: None)
+    mark("start")
     if nv > 0:
         # K goes straight into its cache slot; Q is roped into a scratch copy
         pb.pevlm_rope_qk(s, q[:nv], k[:nv], buf.q_video, buf.k_cache[:nv], 0, nv)
+        mark("rope_video")
         pb.pevlm_assemble_kv(s, None, v[:nv], None, None, buf.k_cache, buf.v_cache)
+        mark("assemble_video")
         pb.pevlm_parallel_prefill_attn(s, buf.q_video, buf.k_cache[:nv], buf.v_cache[:nv], buf.o_video,
                                        buf.lse_video, buf.ws_prefill)
+        mark("prefill_attn")
     if Q > 0:
         pb.pevlm_rope_qk(s, q[nv:], k[nv:], buf.q_question, buf.k_cache[nv:], nv, Q)
+        mark("rope_question")
         pb.pevlm_assemble_kv(s, None, None, None, v[nv:], buf.k_cache, buf.v_cache)
+        mark("assemble_question")
         pb.pevlm_query_attn(s, buf.q_question, buf.k_cache, buf.v_cache, buf.o_question, buf.lse_question,
                             buf.ws_query)
+        mark("query_attn")
     return buf

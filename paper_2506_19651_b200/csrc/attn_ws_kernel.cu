@@ -1,0 +1,481 @@
+// Warp-specialised block-masked flash attention for sm_100a (Eq. 1 under the masks of Eq. 3-5).
+//
+// One CTA owns TWO query tiles of 128 rows that share a kv head and a key-tile list (two q
+// heads of one GQA group at the same block position, or two neighbouring positions), so every
+// K/V tile staged in shared memory feeds both.  Roles (16 warps):
+//   warps 0-3   softmax of query tile 0: one thread per row, scores read from TMEM, running
+//               max/sum in fp32, probabilities written back to TMEM as bf16 over the scores
+//   warps 4-7   softmax of query tile 1
+//   warps 8-11  correction: rescales the O accumulator in TMEM when a row's reference maximum
+//               moved, and writes the normalised output and LSE at the end
+//   warp 12     issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
+//               O += P V (P from TMEM, V from shared memory), ping-ponging between the tiles
+//   warp 13     TMA producer: Q once, then K/V tiles through a 4-slot ring
+// TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
+// Every wait is bounded; an expired wait records PEVLM_ETIMEOUT and the CTA still runs to its
+// normal end (waits become short), so TMEM is always released.
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace pevlm {
+
+constexpr int kWsThreads = 512;
+constexpr int kRing = 4;
+constexpr float kRescaleThresholdLog2 = 8.0f;  // rescale O only when the row maximum grew by > 2^8
+
+enum WsWaitId : int {
+    kWsWaitQ = 11, kWsWaitFull = 12, kWsWaitEmpty = 13, kWsWaitS = 14, kWsWaitAlpha = 15,
+    kWsWaitPO = 16, kWsWaitPV = 17, kWsWaitFinal = 18
+};
+
+template <int D>
+struct WsSmem {
+    static constexpr int kPanels = D / 64;
+    static constexpr int kPanelBytes = kTile * 128;
+    static constexpr int kTileBytes = kPanels * kPanelBytes;
+    static constexpr int kQ0 = 0;
+    static constexpr int kQ1 = kTileBytes;
+    static constexpr int kRing0 = 2 * kTileBytes;
+    static constexpr int kTotal = kRing0 + kRing * kTileBytes;
+};
+
+size_t attn_ws_smem_bytes(int head_dim) {
+    return 1024 + (head_dim == 128 ? WsSmem<128>::kTotal : WsSmem<64>::kTotal);
+}
+
+struct WsSlot {
+    int valid;
+    int q_tok0, q_head0, rows_valid, limit0, b_end, nt;
+};
+struct WsItem {
+    int kv_head, row_div, a_end, b_start, na, split;
+    WsSlot s[2];
+};
+
+__device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ void decode_ws_item(const AttnParams& p, int w, WsItem& it) {
+    it.split = 0;
+    if (p.mode == 0) {
+        it.row_div = 1;
+        int seg_start, seg_len, tiles, pi, g;
+        if (w < p.items_block) {
+            const int combo = w / p.pairs_block;
+            pi = w % p.pairs_block;
+            const int blk = combo / p.Hkv;
+            g = combo % p.Hkv;
+            seg_start = p.S + blk * p.B;
+            seg_len = p.B;
+            tiles = p.tiles_block;
+            it.a_end = p.S;
+        } else {
+            const int w2 = w - p.items_block;
+            g = w2 / p.pairs_sink;
+            pi = w2 % p.pairs_sink;
+            seg_start = 0;
+            seg_len = p.S;
+            tiles = p.tiles_sink;
+            it.a_end = 0;
+        }
+        it.kv_head = g;
+        it.b_start = seg_start;
+        it.na = cdiv(it.a_end, kTile);
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int e = 2 * pi + x;
+            WsSlot& s = it.s[x];
+            s.valid = e < p.G * tiles;
+            const int qt = tiles - 1 - e / p.G;  // heaviest query tiles first
+            s.q_tok0 = seg_start + qt * kTile;
+            s.q_head0 = g * p.G + e % p.G;
+            s.rows_valid = min(kTile, seg_len - qt * kTile);
+            s.limit0 = s.q_tok0;
+            s.b_end = min(s.q_tok0 + kTile, seg_start + seg_len);
+            s.nt = s.valid ? it.na + cdiv(s.b_end - it.b_start, kTile) : 0;
+        }
+    } else {
+        it.split = w % p.n_splits;
+        const int rest = w / p.n_splits;
+        const int q_pairs = cdiv(p.q_tiles, 2);
+        const int pi = rest % q_pairs;
+        const int g = rest / q_pairs;
+        it.kv_head = g;
+        it.row_div = p.G;
+        it.a_end = 0;
+        it.na = 0;
+        const int split_lo = it.split * p.tiles_per_split * kTile;
+        const int split_hi = split_lo + p.tiles_per_split * kTile;
+        it.b_start = split_lo;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int qt = 2 * pi + x;
+            WsSlot& s = it.s[x];
+            s.valid = qt < p.q_tiles;
+            const int tok0 = qt * p.tok_per_tile;
+            const int ntok = max(0, min(p.tok_per_tile, p.Q - tok0));
+            s.q_tok0 = tok0;
+            s.q_head0 = g * p.G;
+            s.rows_valid = ntok * p.G;
+            s.limit0 = p.n_video + tok0;
+            const int kv_end = p.n_video + tok0 + ntok;  // keys past the last row's limit are never visible
+            s.b_end = min(kv_end, split_hi);
+            s.nt = (s.valid && s.b_end > split_lo) ? cdiv(s.b_end - split_lo, kTile) : 0;
+        }
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWsThreads, 1)
+attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap tmap_q,
+               const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+    using L = WsSmem<D>;
+    constexpr int NP = L::kPanels;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[1 + 2 * kRing + 10];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ float s_alpha[2][kTile];
+    __shared__ float s_final_l[2][kTile];
+    __shared__ float s_final_m[2][kTile];
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_q = smem_u32(&bars[0]);
+    const uint32_t bar_full = smem_u32(&bars[1]);
+    const uint32_t bar_empty = smem_u32(&bars[1 + kRing]);
+    const uint32_t bar_s_full = smem_u32(&bars[1 + 2 * kRing]);   // [2]
+    const uint32_t bar_alpha = bar_s_full + 16;                  // [2]
+    const uint32_t bar_po = bar_s_full + 32;                     // [2]
+    const uint32_t bar_pv = bar_s_full + 48;                     // [2]
+    const uint32_t bar_final = bar_s_full + 64;                  // [2]
+
+    if (tid == 0) abort_flag = p.hdr->status;
+    __syncthreads();
+    if (abort_flag != 0) return;
+
+    WsItem it;
+    decode_ws_item(p, blockIdx.x, it);
+    const int nt0 = it.s[0].nt, nt1 = it.s[1].nt;
+    const int nt_max = max(nt0, nt1);
+
+    auto give_up = [&](int which) {
+        if (atomicCAS(&p.hdr->status, 0, PEVLM_ETIMEOUT) == 0) p.hdr->detail = which * 1000000 + blockIdx.x;
+    };
+    auto wait = [&](uint32_t bar, uint32_t parity, int which) {
+        if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
+    };
+    // rows of a slot with no visible key in this CTA's key range (question mode only)
+    auto write_neutral_partial = [&](const WsSlot& s, int row) {
+        if (p.mode == 1 && s.valid && row < s.rows_valid) {
+            const int tok = s.q_tok0 + row / it.row_div;
+            const int head = s.q_head0 + row % it.row_div;
+            const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+            p.part_lse[r] = -INFINITY;
+            float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+            for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    if (nt_max == 0) {
+        if (warp >= 8 && warp < 12) {
+            write_neutral_partial(it.s[0], tid - 256);
+            write_neutral_partial(it.s[1], tid - 256);
+        }
+        return;
+    }
+
+    if (tid == 0) {
+        mbar_init(bar_q, 1);
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(bar_s_full + 8 * x, 1);
+            mbar_init(bar_alpha + 8 * x, kTile);
+            mbar_init(bar_po + 8 * x, 2 * kTile);
+            mbar_init(bar_pv + 8 * x, 1);
+            mbar_init(bar_final + 8 * x, kTile);
+        }
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_q);
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+    }
+    if (warp == 12) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    // key tile j of slot x: first the shared range [0, a_end), then the own range from b_start
+    auto tile_start = [&](int j) { return j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile; };
+    auto tile_valid = [&](const WsSlot& s, int j) {
+        return j < it.na ? min(kTile, it.a_end - j * kTile) : min(kTile, s.b_end - (it.b_start + (j - it.na) * kTile));
+    };
+
+    if (warp == 13) {
+        // ------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            const int q_slots = (it.s[0].valid ? 1 : 0) + (it.s[1].valid ? 1 : 0);
+            mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(q_slots * NP * p.q_box_rows * 128));
+            for (int x = 0; x < 2; ++x)
+                if (it.s[x].valid)
+                    for (int h = 0; h < NP; ++h)
+                        tma_load_3d(smem_base + (x ? L::kQ1 : L::kQ0) + h * L::kPanelBytes, &tmap_q, h * 64,
+                                    it.s[x].q_head0, it.s[x].q_tok0, bar_q);
+            for (int j = 0; j < nt_max; ++j) {
+                const int j0 = tile_start(j);
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+                    const int idx = 2 * j + kv, slot = idx % kRing, use = idx / kRing;
+                    if (use > 0) wait(bar_empty + 8 * slot, (use - 1) & 1, kWsWaitEmpty);
+                    mbar_arrive_expect_tx(bar_full + 8 * slot, L::kTileBytes);
+                    for (int h = 0; h < NP; ++h)
+                        tma_load_3d(smem_base + L::kRing0 + slot * L::kTileBytes + h * L::kPanelBytes,
+                                    kv ? &tmap_v : &tmap_k, h * 64, it.kv_head, j0, bar_full + 8 * slot);
+                }
+            }
+        }
+    } else if (warp == 12) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + (idx % kRing) * L::kTileBytes; };
+            auto wait_full = [&](int idx) { wait(bar_full + 8 * (idx % kRing), (idx / kRing) & 1, kWsWaitFull); };
+            auto issue_qk = [&](int x, int j) {
+                const int n_mma = (tile_valid(it.s[x], j) + 15) & ~15;
+                const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
+                const uint32_t sq = smem_base + (x ? L::kQ1 : L::kQ0), sk = ring_addr(2 * j);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks / 4) * L::kPanelBytes + (ks % 4) * 32;
+                    mma_ss(tmem_base + x * 128, make_smem_desc_sw128(sq + off, 16, 1024),
+                           make_smem_desc_sw128(sk + off, 16, 1024), idesc, ks > 0);
+                }
+                mma_commit(bar_s_full + 8 * x);
+            };
+            auto issue_pv = [&](int x, int j) {
+                const int ksteps = (tile_valid(it.s[x], j) + 15) >> 4;
+                const uint32_t idesc = make_idesc_bf16(kTile, D, true);
+                const uint32_t sv = ring_addr(2 * j + 1);
+                for (int ks = 0; ks < ksteps; ++ks)
+                    mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + ks * 8,
+                           make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc, (j > 0) || (ks > 0));
+                mma_commit(bar_pv + 8 * x);
+            };
+            wait(bar_q, 0, kWsWaitQ);
+            tc_fence_after_sync();
+            for (int j = 0; j <= nt_max; ++j) {
+                if (j < nt_max) {
+                    wait_full(2 * j);
+                    tc_fence_after_sync();
+                    if (j < nt0) issue_qk(0, j);
+                }
+                if (j > 0) {
+                    if (j - 1 < nt1) {
+                        wait_full(2 * (j - 1) + 1);
+                        wait(bar_po + 8, (j - 1) & 1, kWsWaitPO);
+                        tc_fence_after_sync();
+                        issue_pv(1, j - 1);
+                    }
+                    mma_commit(bar_empty + 8 * ((2 * (j - 1) + 1) % kRing));  // V(j-1) consumed
+                }
+                if (j < nt_max) {
+                    if (j < nt1) issue_qk(1, j);
+                    mma_commit(bar_empty + 8 * ((2 * j) % kRing));  // K(j) consumed
+                    if (j < nt0) {
+                        wait_full(2 * j + 1);
+                        wait(bar_po, j & 1, kWsWaitPO);
+                        tc_fence_after_sync();
+                        issue_pv(0, j);
+                    }
+                }
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------- softmax of slot x
+        const int x = warp >> 2;
+        const WsSlot& s = it.s[x];
+        const int row = tid & 127;
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + x * 128 + lane_off;
+        const int my_limit = s.limit0 + row / it.row_div;
+        float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
+        float l_run = 0.f;
+        for (int j = 0; j < s.nt; ++j) {
+            const int j0 = tile_start(j);
+            const int nvalid = tile_valid(s, j);
+            const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > s.limit0);
+            const int max_col = need_mask ? min(nvalid, my_limit - j0 + 1) : kTile;
+            wait(bar_s_full + 8 * x, j & 1, kWsWaitS);
+            tc_fence_after_sync();
+            // pass 1: row maximum
+            float m_tile = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tS + c * 32, r);
+                tmem_wait_ld();
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c * 32 + i < max_col) m_tile = fmaxf(m_tile, __uint_as_float(r[i]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) m_tile = fmaxf(m_tile, __uint_as_float(r[i]));
+                }
+            }
+            float alpha = 1.f;
+            if ((m_tile - m_ref) * p.scale_log2 > kRescaleThresholdLog2 || m_ref == -INFINITY) {
+                const float m_new = fmaxf(m_ref, m_tile);
+                alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
+                m_ref = m_new;
+            }
+            s_alpha[x][row] = alpha;
+            mbar_arrive(bar_alpha + 8 * x);
+            const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
+            // pass 2: probabilities, written over the scores as bf16 pairs (columns [0, 64))
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tS + c * 32, r);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), p.scale_log2, neg_ms));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), p.scale_log2, neg_ms));
+                    if (need_mask) {
+                        if (c * 32 + 2 * i >= max_col) p0 = 0.f;
+                        if (c * 32 + 2 * i + 1 >= max_col) p1 = 0.f;
+                    }
+                    sum += p0 + p1;
+                    pk[i] = pack_bf16x2(p0, p1);
+                }
+                // chunk c of P lands on score columns [16c, 16c+16): already consumed by this
+                // thread (chunks <= c were read before), other rows live in other lanes
+                tmem_st16(tS + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar_po + 8 * x);
+            l_run = l_run * alpha + sum;
+        }
+        s_final_l[x][row] = l_run;
+        s_final_m[x][row] = m_ref;
+        mbar_arrive(bar_final + 8 * x);
+    } else if (warp < 12) {
+        // ------------------------------------------------------------- correction + epilogue
+        const int row = tid & 127;
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        for (int j = 0; j < nt_max; ++j) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                if (j >= it.s[x].nt) continue;
+                wait(bar_alpha + 8 * x, j & 1, kWsWaitAlpha);
+                const float alpha = s_alpha[x][row];
+                if (j > 0) {
+                    wait(bar_pv + 8 * x, (j - 1) & 1, kWsWaitPV);
+                    tc_fence_after_sync();
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                        const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                tc_fence_before_sync();
+                mbar_arrive(bar_po + 8 * x);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const WsSlot& s = it.s[x];
+            if (!s.valid) continue;
+            if (s.nt == 0) {
+                write_neutral_partial(s, row);
+                continue;
+            }
+            wait(bar_final + 8 * x, 0, kWsWaitFinal);
+            wait(bar_pv + 8 * x, (s.nt - 1) & 1, kWsWaitPV);
+            tc_fence_after_sync();
+            const float l = s_final_l[x][row], m = s_final_m[x][row];
+            const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+            const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
+            const bool row_ok = row < s.rows_valid;
+            const int tok = s.q_tok0 + row / it.row_div;
+            const int head = s.q_head0 + row % it.row_div;
+            const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                tmem_wait_ld();
+                if (!row_ok) continue;
+                if (p.mode == 0) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            w[e] = pack_bf16x2(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
+                                               __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
+                        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                } else {
+                    const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                    float4* dst = reinterpret_cast<float4*>(p.part_o + r * D + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
+                                             __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                }
+            }
+            if (row_ok) {
+                if (p.mode == 0) {
+                    if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
+                } else {
+                    p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 12) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+cudaError_t launch_attn_ws(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
+                           const CUtensorMap& tv, cudaStream_t stream) {
+    if (p.n_items <= 0) return cudaSuccess;
+    const size_t smem = attn_ws_smem_bytes(head_dim);
+    cudaError_t e;
+    if (head_dim == 128) {
+        e = cudaFuncSetAttribute(attn_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        attn_ws_kernel<128><<<p.n_items, kWsThreads, smem, stream>>>(p, tq, tk, tv);
+    } else {
+        e = cudaFuncSetAttribute(attn_ws_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        attn_ws_kernel<64><<<p.n_items, kWsThreads, smem, stream>>>(p, tq, tk, tv);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace pevlm

@@ -218,7 +218,10 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         return j < it.na ? min(kTile, it.a_end - j * kTile) : min(kTile, s.b_end - (it.b_start + (j - it.na) * kTile));
     };
 
-    if (warp == 13) {
+    // register budget per warpgroup: 2 x 192 (softmax) + 80 (correction) + 48 (TMA/MMA) = 512 x 128
+    if (warp >= 12) {
+        reg_dealloc<48>();
+      if (warp == 13) {
         // ------------------------------------------------------------- TMA producer
         if (lane == 0) {
             const int q_slots = (it.s[0].valid ? 1 : 0) + (it.s[1].valid ? 1 : 0);
@@ -241,7 +244,7 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                 }
             }
         }
-    } else if (warp == 12) {
+      } else if (warp == 12) {
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + (idx % kRing) * L::kTileBytes; };
@@ -296,8 +299,10 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                 }
             }
         }
+      }
     } else if (warp < 8) {
         // ------------------------------------------------------------- softmax of slot x
+        reg_alloc<192>();
         const int x = warp >> 2;
         const WsSlot& s = it.s[x];
         const int row = tid & 127;
@@ -313,22 +318,24 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
             const int max_col = need_mask ? min(nvalid, my_limit - j0 + 1) : kTile;
             wait(bar_s_full + 8 * x, j & 1, kWsWaitS);
             tc_fence_after_sync();
-            // pass 1: row maximum
-            float m_tile = -INFINITY;
+            // all 128 scores of the row in registers: one round trip to TMEM
+            uint32_t r[128];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tS + c * 32, r);
-                tmem_wait_ld();
-                if (need_mask) {
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
+            tmem_wait_ld();
+            if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c * 32 + i < max_col) m_tile = fmaxf(m_tile, __uint_as_float(r[i]));
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) m_tile = fmaxf(m_tile, __uint_as_float(r[i]));
-                }
+                for (int i = 0; i < 128; ++i)
+                    if (i >= max_col) r[i] = 0xff800000u;  // -inf
             }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < 128; i += 8) {
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+                    mx[a] = fmax3(mx[a], __uint_as_float(r[i + 2 * a]), __uint_as_float(r[i + 2 * a + 1]));
+            }
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             float alpha = 1.f;
             if ((m_tile - m_ref) * p.scale_log2 > kRescaleThresholdLog2 || m_ref == -INFINITY) {
                 const float m_new = fmaxf(m_ref, m_tile);
@@ -338,29 +345,21 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
             s_alpha[x][row] = alpha;
             mbar_arrive(bar_alpha + 8 * x);
             const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
-            // pass 2: probabilities, written over the scores as bf16 pairs (columns [0, 64))
-            float sum = 0.f;
+            // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot)
+            float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tS + c * 32, r);
-                tmem_wait_ld();
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), p.scale_log2, neg_ms));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), p.scale_log2, neg_ms));
-                    if (need_mask) {
-                        if (c * 32 + 2 * i >= max_col) p0 = 0.f;
-                        if (c * 32 + 2 * i + 1 >= max_col) p1 = 0.f;
-                    }
-                    sum += p0 + p1;
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i]), p.scale_log2, neg_ms));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i + 1]), p.scale_log2, neg_ms));
+                    sm[i & 3] += p0 + p1;
                     pk[i] = pack_bf16x2(p0, p1);
                 }
-                // chunk c of P lands on score columns [16c, 16c+16): already consumed by this
-                // thread (chunks <= c were read before), other rows live in other lanes
                 tmem_st16(tS + c * 16, pk);
             }
+            const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar_po + 8 * x);
@@ -369,8 +368,9 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         s_final_l[x][row] = l_run;
         s_final_m[x][row] = m_ref;
         mbar_arrive(bar_final + 8 * x);
-    } else if (warp < 12) {
+    } else {
         // ------------------------------------------------------------- correction + epilogue
+        reg_dealloc<80>();
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         for (int j = 0; j < nt_max; ++j) {

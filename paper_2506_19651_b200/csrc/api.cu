@@ -272,6 +272,10 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
         if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         p.o = static_cast<__nv_bfloat16*>(o) + qoff;
         p.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * nv : nullptr;
+        if (b > 0) {  // every launch starts its work counter at zero; the status word is kept
+            e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
+            if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
+        }
         e = simple ? launch_attn(p, d, tq, tk, tv, st) : launch_attn_ws(p, d, tq, tk, tv, st);
         if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
     }
@@ -322,6 +326,10 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
         p.part_o = part;
         p.part_lse = part + static_cast<size_t>(p.n_splits) * p.Q * p.Hq * d;
         const int64_t qoff = static_cast<int64_t>(b) * p.Q * p.Hq * d, koff = static_cast<int64_t>(b) * L * p.Hkv * d;
+        if (b > 0) {
+            e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
+            if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
+        }
         CUtensorMap tq, tk, tv;
         if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;

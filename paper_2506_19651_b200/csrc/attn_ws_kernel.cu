@@ -10,7 +10,11 @@
 //               moved, and writes the normalised output and LSE at the end
 //   warp 12     issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
 //               O += P V (P from TMEM, V from shared memory), ping-ponging between the tiles
-//   warp 13     TMA producer: Q once, then K/V tiles through a 4-slot ring
+//   warp 13     work scheduler and TMA producer: takes the next work item from a global
+//               counter, publishes it to the other roles, loads its two Q tiles, then streams
+//               K/V tiles through a 4-slot ring that runs on across items
+// The kernel is persistent (one CTA per SM): while the correction warps write out item k, the
+// producer, the MMA warp and the softmax warps already work on item k+1.
 // TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
 // Every wait is bounded; an expired wait records PEVLM_ETIMEOUT and the CTA still runs to its
 // normal end (waits become short), so TMEM is always released.
@@ -25,7 +29,8 @@ constexpr float kRescaleThresholdLog2 = 8.0f;  // rescale O only when the row ma
 
 enum WsWaitId : int {
     kWsWaitQ = 11, kWsWaitFull = 12, kWsWaitEmpty = 13, kWsWaitS = 14, kWsWaitAlpha = 15,
-    kWsWaitPO = 16, kWsWaitPV = 17, kWsWaitFinal = 18
+    kWsWaitPO = 16, kWsWaitPV = 17, kWsWaitFinal = 18, kWsWaitItem = 19, kWsWaitItemFree = 20,
+    kWsWaitQFree = 21, kWsWaitOFree = 22
 };
 
 template <int D>
@@ -131,72 +136,44 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
     using L = WsSmem<D>;
     constexpr int NP = L::kPanels;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[1 + 2 * kRing + 10];
+    // barrier map (uint64 each): [0,2) item_full  [2,4) item_free  [4,6) q_full  [6,8) q_free
+    // [8,12) ring full  [12,16) ring empty  then per slot x: s_full, alpha, po, pv, final, o_free
+    __shared__ uint64_t bars[16 + 12];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int s_item[2];
     __shared__ float s_alpha[2][kTile];
-    __shared__ float s_final_l[2][kTile];
-    __shared__ float s_final_m[2][kTile];
+    __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a one-tile
+    __shared__ float s_final_m[2][2][kTile];  // item while the previous item's epilogue is still running
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_q = smem_u32(&bars[0]);
-    const uint32_t bar_full = smem_u32(&bars[1]);
-    const uint32_t bar_empty = smem_u32(&bars[1 + kRing]);
-    const uint32_t bar_s_full = smem_u32(&bars[1 + 2 * kRing]);   // [2]
-    const uint32_t bar_alpha = bar_s_full + 16;                  // [2]
-    const uint32_t bar_po = bar_s_full + 32;                     // [2]
-    const uint32_t bar_pv = bar_s_full + 48;                     // [2]
-    const uint32_t bar_final = bar_s_full + 64;                  // [2]
-
-    if (tid == 0) abort_flag = p.hdr->status;
-    __syncthreads();
-    if (abort_flag != 0) return;
-
-    WsItem it;
-    decode_ws_item(p, blockIdx.x, it);
-    const int nt0 = it.s[0].nt, nt1 = it.s[1].nt;
-    const int nt_max = max(nt0, nt1);
-
-    auto give_up = [&](int which) {
-        if (atomicCAS(&p.hdr->status, 0, PEVLM_ETIMEOUT) == 0) p.hdr->detail = which * 1000000 + blockIdx.x;
-    };
-    auto wait = [&](uint32_t bar, uint32_t parity, int which) {
-        if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
-    };
-    // rows of a slot with no visible key in this CTA's key range (question mode only)
-    auto write_neutral_partial = [&](const WsSlot& s, int row) {
-        if (p.mode == 1 && s.valid && row < s.rows_valid) {
-            const int tok = s.q_tok0 + row / it.row_div;
-            const int head = s.q_head0 + row % it.row_div;
-            const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-            p.part_lse[r] = -INFINITY;
-            float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
-            for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    };
-    if (nt_max == 0) {
-        if (warp >= 8 && warp < 12) {
-            write_neutral_partial(it.s[0], tid - 256);
-            write_neutral_partial(it.s[1], tid - 256);
-        }
-        return;
-    }
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    const uint32_t bar_item_full = bar0, bar_item_free = bar0 + 16, bar_q_full = bar0 + 32, bar_q_free = bar0 + 48;
+    const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
+    const uint32_t bar_s_full = bar0 + 128, bar_alpha = bar0 + 144, bar_po = bar0 + 160, bar_pv = bar0 + 176;
+    const uint32_t bar_final = bar0 + 192, bar_o_free = bar0 + 208;
+    constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA lane + two softmax warpgroups + correction warpgroup
 
     if (tid == 0) {
-        mbar_init(bar_q, 1);
+        abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_item_full + 8 * i, 1);
+            mbar_init(bar_item_free + 8 * i, kItemConsumers);
+            mbar_init(bar_q_full + 8 * i, 1);
+            mbar_init(bar_q_free + 8 * i, 1);
+            mbar_init(bar_s_full + 8 * i, 1);
+            mbar_init(bar_alpha + 8 * i, kTile);
+            mbar_init(bar_po + 8 * i, 2 * kTile);
+            mbar_init(bar_pv + 8 * i, 1);
+            mbar_init(bar_final + 8 * i, kTile);
+            mbar_init(bar_o_free + 8 * i, kTile);
+        }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(bar_full + 8 * i, 1);
             mbar_init(bar_empty + 8 * i, 1);
-        }
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(bar_s_full + 8 * x, 1);
-            mbar_init(bar_alpha + 8 * x, kTile);
-            mbar_init(bar_po + 8 * x, 2 * kTile);
-            mbar_init(bar_pv + 8 * x, 1);
-            mbar_init(bar_final + 8 * x, kTile);
         }
         fence_mbar_init();
         tma_prefetch_desc(&tmap_q);
@@ -212,9 +189,22 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
 
-    // key tile j of slot x: first the shared range [0, a_end), then the own range from b_start
-    auto tile_start = [&](int j) { return j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile; };
-    auto tile_valid = [&](const WsSlot& s, int j) {
+    auto give_up = [&](int which) {
+        if (atomicCAS(&p.hdr->status, 0, PEVLM_ETIMEOUT) == 0) p.hdr->detail = which * 1000000 + blockIdx.x;
+    };
+    auto wait = [&](uint32_t bar, uint32_t parity, int which) {
+        if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
+    };
+    // consumer side of the item queue: k-th item of this CTA, -1 = no more work
+    auto next_item = [&](int k) {
+        wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWsWaitItem);
+        const int w = s_item[k & 1];
+        mbar_arrive(bar_item_free + 8 * (k & 1));
+        return w;
+    };
+    // key tile j of an item: first the shared range [0, a_end), then the own range from b_start
+    auto tile_start = [&](const WsItem& it, int j) { return j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile; };
+    auto tile_valid = [&](const WsItem& it, const WsSlot& s, int j) {
         return j < it.na ? min(kTile, it.a_end - j * kTile) : min(kTile, s.b_end - (it.b_start + (j - it.na) * kTile));
     };
 
@@ -222,80 +212,122 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
     if (warp >= 12) {
         reg_dealloc<48>();
       if (warp == 13) {
-        // ------------------------------------------------------------- TMA producer
+        // ------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
-            const int q_slots = (it.s[0].valid ? 1 : 0) + (it.s[1].valid ? 1 : 0);
-            mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(q_slots * NP * p.q_box_rows * 128));
-            for (int x = 0; x < 2; ++x)
-                if (it.s[x].valid)
+            int ring_idx = 0;          // K/V tiles loaded so far (ring position), runs on across items
+            int q_loads[2] = {0, 0};   // Q loads per slot so far
+            for (int k = 0;; ++k) {
+                int w = (k == 0) ? static_cast<int>(blockIdx.x)
+                                 : static_cast<int>(gridDim.x) + atomicAdd(&p.hdr->work_counter, 1);
+                if (w >= p.n_items || abort_flag != 0 || *reinterpret_cast<volatile int32_t*>(&p.hdr->status) != 0) w = -1;
+                if (k >= 2) wait(bar_item_free + 8 * (k & 1), ((k >> 1) - 1) & 1, kWsWaitItemFree);
+                s_item[k & 1] = w;
+                mbar_arrive(bar_item_full + 8 * (k & 1));
+                if (w < 0) break;
+                WsItem it;
+                decode_ws_item(p, w, it);
+                const int nt_max = max(it.s[0].nt, it.s[1].nt);
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    if (it.s[x].nt == 0) continue;
+                    if (q_loads[x] > 0) wait(bar_q_free + 8 * x, (q_loads[x] - 1) & 1, kWsWaitQFree);
+                    mbar_arrive_expect_tx(bar_q_full + 8 * x, static_cast<uint32_t>(NP * p.q_box_rows * 128));
                     for (int h = 0; h < NP; ++h)
                         tma_load_3d(smem_base + (x ? L::kQ1 : L::kQ0) + h * L::kPanelBytes, &tmap_q, h * 64,
-                                    it.s[x].q_head0, it.s[x].q_tok0, bar_q);
-            for (int j = 0; j < nt_max; ++j) {
-                const int j0 = tile_start(j);
+                                    it.s[x].q_head0, it.s[x].q_tok0, bar_q_full + 8 * x);
+                    ++q_loads[x];
+                }
+                for (int j = 0; j < nt_max; ++j) {
+                    const int j0 = tile_start(it, j);
 #pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
-                    const int idx = 2 * j + kv, slot = idx % kRing, use = idx / kRing;
-                    if (use > 0) wait(bar_empty + 8 * slot, (use - 1) & 1, kWsWaitEmpty);
-                    mbar_arrive_expect_tx(bar_full + 8 * slot, L::kTileBytes);
-                    for (int h = 0; h < NP; ++h)
-                        tma_load_3d(smem_base + L::kRing0 + slot * L::kTileBytes + h * L::kPanelBytes,
-                                    kv ? &tmap_v : &tmap_k, h * 64, it.kv_head, j0, bar_full + 8 * slot);
+                    for (int kv = 0; kv < 2; ++kv) {
+                        const int slot = ring_idx % kRing, use = ring_idx / kRing;
+                        if (use > 0) wait(bar_empty + 8 * slot, (use - 1) & 1, kWsWaitEmpty);
+                        mbar_arrive_expect_tx(bar_full + 8 * slot, L::kTileBytes);
+                        for (int h = 0; h < NP; ++h)
+                            tma_load_3d(smem_base + L::kRing0 + slot * L::kTileBytes + h * L::kPanelBytes,
+                                        kv ? &tmap_v : &tmap_k, h * 64, it.kv_head, j0, bar_full + 8 * slot);
+                        ++ring_idx;
+                    }
                 }
             }
         }
       } else if (warp == 12) {
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + (idx % kRing) * L::kTileBytes; };
-            auto wait_full = [&](int idx) { wait(bar_full + 8 * (idx % kRing), (idx / kRing) & 1, kWsWaitFull); };
-            auto issue_qk = [&](int x, int j) {
-                const int n_mma = (tile_valid(it.s[x], j) + 15) & ~15;
-                const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
-                const uint32_t sq = smem_base + (x ? L::kQ1 : L::kQ0), sk = ring_addr(2 * j);
+            int ring_base = 0;        // ring position of this item's K(0)
+            int cnt[2] = {0, 0};      // tiles issued per slot so far (phase of s_full / po / pv)
+            int q_uses[2] = {0, 0};   // items in which the slot was active so far
+            for (int k = 0;; ++k) {
+                const int w = next_item(k);
+                if (w < 0) break;
+                WsItem it;
+                decode_ws_item(p, w, it);
+                const int nt0 = it.s[0].nt, nt1 = it.s[1].nt;
+                const int nt_max = max(nt0, nt1);
+                auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
+                auto wait_full = [&](int idx) {
+                    const int g = ring_base + idx;
+                    wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWsWaitFull);
+                };
+                auto commit_empty = [&](int idx) { mma_commit(bar_empty + 8 * ((ring_base + idx) % kRing)); };
+                auto issue_qk = [&](int x, int j) {
+                    const int n_mma = (tile_valid(it, it.s[x], j) + 15) & ~15;
+                    const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
+                    const uint32_t sq = smem_base + (x ? L::kQ1 : L::kQ0), sk = ring_addr(2 * j);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * L::kPanelBytes + (ks % 4) * 32;
-                    mma_ss(tmem_base + x * 128, make_smem_desc_sw128(sq + off, 16, 1024),
-                           make_smem_desc_sw128(sk + off, 16, 1024), idesc, ks > 0);
-                }
-                mma_commit(bar_s_full + 8 * x);
-            };
-            auto issue_pv = [&](int x, int j) {
-                const int ksteps = (tile_valid(it.s[x], j) + 15) >> 4;
-                const uint32_t idesc = make_idesc_bf16(kTile, D, true);
-                const uint32_t sv = ring_addr(2 * j + 1);
-                for (int ks = 0; ks < ksteps; ++ks)
-                    mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + ks * 8,
-                           make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc, (j > 0) || (ks > 0));
-                mma_commit(bar_pv + 8 * x);
-            };
-            wait(bar_q, 0, kWsWaitQ);
-            tc_fence_after_sync();
-            for (int j = 0; j <= nt_max; ++j) {
-                if (j < nt_max) {
-                    wait_full(2 * j);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = (ks / 4) * L::kPanelBytes + (ks % 4) * 32;
+                        mma_ss(tmem_base + x * 128, make_smem_desc_sw128(sq + off, 16, 1024),
+                               make_smem_desc_sw128(sk + off, 16, 1024), idesc, ks > 0);
+                    }
+                    mma_commit(bar_s_full + 8 * x);
+                    if (j == it.s[x].nt - 1) mma_commit(bar_q_free + 8 * x);  // last use of this Q tile
+                };
+                auto issue_pv = [&](int x, int j) {
+                    wait(bar_po + 8 * x, (cnt[x] + j) & 1, kWsWaitPO);
+                    // the previous item's output must have left TMEM before O is overwritten
+                    if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWsWaitOFree);
                     tc_fence_after_sync();
-                    if (j < nt0) issue_qk(0, j);
-                }
-                if (j > 0) {
-                    if (j - 1 < nt1) {
-                        wait_full(2 * (j - 1) + 1);
-                        wait(bar_po + 8, (j - 1) & 1, kWsWaitPO);
+                    const int ksteps = (tile_valid(it, it.s[x], j) + 15) >> 4;
+                    const uint32_t idesc = make_idesc_bf16(kTile, D, true);
+                    const uint32_t sv = ring_addr(2 * j + 1);
+                    for (int ks = 0; ks < ksteps; ++ks)
+                        mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + ks * 8,
+                               make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc, (j > 0) || (ks > 0));
+                    mma_commit(bar_pv + 8 * x);
+                };
+#pragma unroll
+                for (int x = 0; x < 2; ++x)
+                    if (it.s[x].nt > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWsWaitQ);
+                tc_fence_after_sync();
+                for (int j = 0; j <= nt_max; ++j) {
+                    if (j < nt_max) {
+                        wait_full(2 * j);
                         tc_fence_after_sync();
-                        issue_pv(1, j - 1);
+                        if (j < nt0) issue_qk(0, j);
                     }
-                    mma_commit(bar_empty + 8 * ((2 * (j - 1) + 1) % kRing));  // V(j-1) consumed
+                    if (j > 0) {
+                        if (j - 1 < nt1) {
+                            wait_full(2 * (j - 1) + 1);
+                            issue_pv(1, j - 1);
+                        }
+                        commit_empty(2 * (j - 1) + 1);  // V(j-1) consumed
+                    }
+                    if (j < nt_max) {
+                        if (j < nt1) issue_qk(1, j);
+                        commit_empty(2 * j);  // K(j) consumed
+                        if (j < nt0) {
+                            wait_full(2 * j + 1);
+                            issue_pv(0, j);
+                        }
+                    }
                 }
-                if (j < nt_max) {
-                    if (j < nt1) issue_qk(1, j);
-                    mma_commit(bar_empty + 8 * ((2 * j) % kRing));  // K(j) consumed
-                    if (j < nt0) {
-                        wait_full(2 * j + 1);
-                        wait(bar_po, j & 1, kWsWaitPO);
-                        tc_fence_after_sync();
-                        issue_pv(0, j);
-                    }
+                ring_base += 2 * nt_max;
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    cnt[x] += it.s[x].nt;
+                    if (it.s[x].nt > 0) ++q_uses[x];
                 }
             }
         }
@@ -304,85 +336,107 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         // ------------------------------------------------------------- softmax of slot x
         reg_alloc<192>();
         const int x = warp >> 2;
-        const WsSlot& s = it.s[x];
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + x * 128 + lane_off;
-        const int my_limit = s.limit0 + row / it.row_div;
-        float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
-        float l_run = 0.f;
-        for (int j = 0; j < s.nt; ++j) {
-            const int j0 = tile_start(j);
-            const int nvalid = tile_valid(s, j);
-            const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > s.limit0);
-            const int max_col = need_mask ? min(nvalid, my_limit - j0 + 1) : kTile;
-            wait(bar_s_full + 8 * x, j & 1, kWsWaitS);
-            tc_fence_after_sync();
-            // all 128 scores of the row in registers: one round trip to TMEM
-            uint32_t r[128];
+        int cnt = 0;   // tiles of this slot processed so far (phase of s_full)
+        int uses = 0;  // items in which this slot was active so far
+        for (int k = 0;; ++k) {
+            const int w = next_item(k);
+            if (w < 0) break;
+            WsItem it;
+            decode_ws_item(p, w, it);
+            const WsSlot& s = it.s[x];
+            if (s.nt == 0) continue;
+            const int my_limit = s.limit0 + row / it.row_div;
+            float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
+            float l_run = 0.f;
+            for (int j = 0; j < s.nt; ++j, ++cnt) {
+                const int j0 = tile_start(it, j);
+                const int nvalid = tile_valid(it, s, j);
+                const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > s.limit0);
+                const int max_col = need_mask ? min(nvalid, my_limit - j0 + 1) : kTile;
+                wait(bar_s_full + 8 * x, cnt & 1, kWsWaitS);
+                tc_fence_after_sync();
+                // all 128 scores of the row in registers: one round trip to TMEM
+                uint32_t r[128];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
-            tmem_wait_ld();
-            if (need_mask) {
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
+                tmem_wait_ld();
+                if (need_mask) {
 #pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i >= max_col) r[i] = 0xff800000u;  // -inf
-            }
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int i = 0; i < 128; i += 8) {
-#pragma unroll
-                for (int a = 0; a < 4; ++a)
-                    mx[a] = fmax3(mx[a], __uint_as_float(r[i + 2 * a]), __uint_as_float(r[i + 2 * a + 1]));
-            }
-            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            float alpha = 1.f;
-            if ((m_tile - m_ref) * p.scale_log2 > kRescaleThresholdLog2 || m_ref == -INFINITY) {
-                const float m_new = fmaxf(m_ref, m_tile);
-                alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
-                m_ref = m_new;
-            }
-            s_alpha[x][row] = alpha;
-            mbar_arrive(bar_alpha + 8 * x);
-            const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
-            // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot)
-            float sm[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i]), p.scale_log2, neg_ms));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i + 1]), p.scale_log2, neg_ms));
-                    sm[i & 3] += p0 + p1;
-                    pk[i] = pack_bf16x2(p0, p1);
+                    for (int i = 0; i < 128; ++i)
+                        if (i >= max_col) r[i] = 0xff800000u;  // -inf
                 }
-                tmem_st16(tS + c * 16, pk);
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int i = 0; i < 128; i += 8) {
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+                        mx[a] = fmax3(mx[a], __uint_as_float(r[i + 2 * a]), __uint_as_float(r[i + 2 * a + 1]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                float alpha = 1.f;
+                if ((m_tile - m_ref) * p.scale_log2 > kRescaleThresholdLog2 || m_ref == -INFINITY) {
+                    const float m_new = fmaxf(m_ref, m_tile);
+                    alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
+                    m_ref = m_new;
+                }
+                if (j > 0) {
+                    s_alpha[x][row] = alpha;
+                    mbar_arrive(bar_alpha + 8 * x);
+                }
+                const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
+                // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot)
+                float sm[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i]), p.scale_log2, neg_ms));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i + 1]), p.scale_log2, neg_ms));
+                        sm[i & 3] += p0 + p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
+                tmem_wait_st();
+                tc_fence_before_sync();
+                // the first tile of an item has no O to correct: this thread also arrives for its
+                // correction partner, so the epilogue of the previous item is not on the MMA's path
+                mbar_arrive_n(bar_po + 8 * x, j == 0 ? 2 : 1);
+                l_run = l_run * alpha + sum;
             }
-            const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
-            tmem_wait_st();
-            tc_fence_before_sync();
-            mbar_arrive(bar_po + 8 * x);
-            l_run = l_run * alpha + sum;
+            s_final_l[uses & 1][x][row] = l_run;
+            s_final_m[uses & 1][x][row] = m_ref;
+            mbar_arrive(bar_final + 8 * x);
+            ++uses;
         }
-        s_final_l[x][row] = l_run;
-        s_final_m[x][row] = m_ref;
-        mbar_arrive(bar_final + 8 * x);
     } else {
         // ------------------------------------------------------------- correction + epilogue
         reg_dealloc<80>();
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        for (int j = 0; j < nt_max; ++j) {
+        int cnt[2] = {0, 0};    // tiles per slot so far (phase of pv; alpha runs one behind per item)
+        int acnt[2] = {0, 0};   // alpha phases per slot so far (tiles with j > 0)
+        int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_free)
+        for (int k = 0;; ++k) {
+            const int w = next_item(k);
+            if (w < 0) break;
+            WsItem it;
+            decode_ws_item(p, w, it);
+            const int nt_max = max(it.s[0].nt, it.s[1].nt);
+            for (int j = 1; j < nt_max; ++j) {
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                if (j >= it.s[x].nt) continue;
-                wait(bar_alpha + 8 * x, j & 1, kWsWaitAlpha);
-                const float alpha = s_alpha[x][row];
-                if (j > 0) {
-                    wait(bar_pv + 8 * x, (j - 1) & 1, kWsWaitPV);
-                    tc_fence_after_sync();
+                for (int x = 0; x < 2; ++x) {
+                    if (j >= it.s[x].nt) continue;
+                    wait(bar_alpha + 8 * x, (acnt[x] + j - 1) & 1, kWsWaitAlpha);
+                    const float alpha = s_alpha[x][row];
                     if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                        wait(bar_pv + 8 * x, (cnt[x] + j - 1) & 1, kWsWaitPV);
+                        tc_fence_after_sync();
                         const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
@@ -395,60 +449,80 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                         }
                         tmem_wait_st();
                     }
+                    tc_fence_before_sync();
+                    mbar_arrive(bar_po + 8 * x);
                 }
-                tc_fence_before_sync();
-                mbar_arrive(bar_po + 8 * x);
             }
-        }
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            const WsSlot& s = it.s[x];
-            if (!s.valid) continue;
-            if (s.nt == 0) {
-                write_neutral_partial(s, row);
-                continue;
-            }
-            wait(bar_final + 8 * x, 0, kWsWaitFinal);
-            wait(bar_pv + 8 * x, (s.nt - 1) & 1, kWsWaitPV);
-            tc_fence_after_sync();
-            const float l = s_final_l[x][row], m = s_final_m[x][row];
-            const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
-            const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
-            const bool row_ok = row < s.rows_valid;
-            const int tok = s.q_tok0 + row / it.row_div;
-            const int head = s.q_head0 + row % it.row_div;
-            const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tO + c * 32, o);
-                tmem_wait_ld();
-                if (!row_ok) continue;
-                if (p.mode == 0) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            w[e] = pack_bf16x2(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
-                                               __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
-                        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int x = 0; x < 2; ++x) {
+                const WsSlot& s = it.s[x];
+                if (!s.valid) continue;
+                const bool row_ok = row < s.rows_valid;
+                const int tok = s.q_tok0 + row / it.row_div;
+                const int head = s.q_head0 + row % it.row_div;
+                if (s.nt == 0) {
+                    // question-mode slot with no visible key in this CTA's key range: neutral partial
+                    if (p.mode == 1 && row_ok) {
+                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                        p.part_lse[r] = -INFINITY;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+                        for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
-                } else {
-                    const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-                    float4* dst = reinterpret_cast<float4*>(p.part_o + r * D + c * 32);
+                    continue;
+                }
+                wait(bar_final + 8 * x, uses[x] & 1, kWsWaitFinal);
+                wait(bar_pv + 8 * x, (cnt[x] + s.nt - 1) & 1, kWsWaitPV);
+                tc_fence_after_sync();
+                const float l = s_final_l[uses[x] & 1][x][row], m = s_final_m[uses[x] & 1][x][row];
+                const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+                const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
+                const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
-                                             __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
+                    if (c == D / 32 - 1) {
+                        // every column of this row is in registers: the accumulator may be reused
+                        tc_fence_before_sync();
+                        mbar_arrive(bar_o_free + 8 * x);
+                    }
+                    if (!row_ok) continue;
+                    if (p.mode == 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t wd[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                wd[e] = pack_bf16x2(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
+                                                    __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
+                            dst[v] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                        }
+                    } else {
+                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D + c * 32);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
+                                                 __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                    }
+                }
+                if (row_ok) {
+                    if (p.mode == 0) {
+                        if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
+                    } else {
+                        p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+                    }
                 }
             }
-            if (row_ok) {
-                if (p.mode == 0) {
-                    if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
-                } else {
-                    p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                const int nt = it.s[x].nt;
+                cnt[x] += nt;
+                if (nt > 0) {
+                    acnt[x] += nt - 1;
+                    ++uses[x];
                 }
             }
         }
@@ -465,15 +539,20 @@ cudaError_t launch_attn_ws(const AttnParams& p, int head_dim, const CUtensorMap&
                            const CUtensorMap& tv, cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
     const size_t smem = attn_ws_smem_bytes(head_dim);
-    cudaError_t e;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int grid = p.n_items < sms ? p.n_items : sms;  // persistent: one CTA per SM
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_ws_kernel<128><<<p.n_items, kWsThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_ws_kernel<128><<<grid, kWsThreads, smem, stream>>>(p, tq, tk, tv);
     } else {
         e = cudaFuncSetAttribute(attn_ws_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_ws_kernel<64><<<p.n_items, kWsThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_ws_kernel<64><<<grid, kWsThreads, smem, stream>>>(p, tq, tk, tv);
     }
     return cudaGetLastError();
 }

@@ -3,13 +3,16 @@
 // One CTA owns TWO query tiles of 128 rows that share a kv head and a key-tile list (two q
 // heads of one GQA group at the same block position, or two neighbouring positions), so every
 // K/V tile staged in shared memory feeds both.  Roles (16 warps):
-//   warps 0-3   softmax of query tile 0: one thread per row, scores read from TMEM, running
-//               max/sum in fp32, probabilities written back to TMEM as bf16 over the scores
+//   warps 0-3   softmax of query tile 0: one thread per row; the 128 scores of a key tile are
+//               read from TMEM once, running max/sum kept in fp32, probabilities written back
+//               over the scores as bf16; the rare rescale of the O accumulator (the reference
+//               maximum moves only when a row's maximum grows by more than 2^8) is done in
+//               place by the same threads
 //   warps 4-7   softmax of query tile 1
-//   warps 8-11  correction: rescales the O accumulator in TMEM when a row's reference maximum
-//               moved, and writes the normalised output and LSE at the end
+//   warps 8-11  epilogue: normalised output and LSE of a finished item, TMEM -> global
 //   warp 12     issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
-//               O += P V (P from TMEM, V from shared memory), ping-ponging between the tiles
+//               O += P V (P from TMEM, V from shared memory), ping-ponging between the two
+//               query tiles so one is in the tensor cores while the other is in its softmax
 //   warp 13     work scheduler and TMA producer: takes the next work item from a global
 //               counter, publishes it to the other roles, loads its two Q tiles, then streams
 //               K/V tiles through a 4-slot ring that runs on across items
@@ -32,6 +35,19 @@ enum WsWaitId : int {
     kWsWaitPO = 16, kWsWaitPV = 17, kWsWaitFinal = 18, kWsWaitItem = 19, kWsWaitItemFree = 20,
     kWsWaitQFree = 21, kWsWaitOFree = 22
 };
+
+// Optional in-kernel cycle accounting (compile with -DPEVLM_PROFILE): CTA 0 accumulates the
+// cycles its MMA thread and one softmax thread spend in each wait / phase and leaves them in
+// the padding of the workspace header.
+#ifdef PEVLM_PROFILE
+#define PROF_DECL(n) long long prof_acc[n] = {}; long long prof_t = clock64();
+#define PROF_LAP(i) { const long long prof_now = clock64(); prof_acc[i] += prof_now - prof_t; prof_t = prof_now; }
+#define PROF_DUMP(base, n) if (blockIdx.x == 0) { for (int prof_i = 0; prof_i < (n); ++prof_i) p.hdr->pad[(base) + prof_i] = static_cast<int32_t>(prof_acc[prof_i] >> 4); }
+#else
+#define PROF_DECL(n)
+#define PROF_LAP(i)
+#define PROF_DUMP(base, n)
+#endif
 
 template <int D>
 struct WsSmem {
@@ -136,14 +152,14 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
     using L = WsSmem<D>;
     constexpr int NP = L::kPanels;
     extern __shared__ uint8_t smem_raw[];
-    // barrier map (uint64 each): [0,2) item_full  [2,4) item_free  [4,6) q_full  [6,8) q_free
-    // [8,12) ring full  [12,16) ring empty  then per slot x: s_full, alpha, po, pv, final, o_free
-    __shared__ uint64_t bars[16 + 12];
+    // barrier map (uint64 each): [0,2) item_full [2,4) item_free [4,6) q_full [6,8) q_free
+    // [8,12) ring full [12,16) ring empty, then per slot x: [16,18) s_full [18,20) po [20,22) pv
+    // [22,24) final [24,26) o_free [26,28) o_done
+    __shared__ uint64_t bars[28];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int s_item[2];
-    __shared__ float s_alpha[2][kTile];
-    __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a one-tile
+    __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a short
     __shared__ float s_final_m[2][2][kTile];  // item while the previous item's epilogue is still running
 
     const int tid = threadIdx.x;
@@ -153,9 +169,9 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
     const uint32_t bar0 = smem_u32(&bars[0]);
     const uint32_t bar_item_full = bar0, bar_item_free = bar0 + 16, bar_q_full = bar0 + 32, bar_q_free = bar0 + 48;
     const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
-    const uint32_t bar_s_full = bar0 + 128, bar_alpha = bar0 + 144, bar_po = bar0 + 160, bar_pv = bar0 + 176;
-    const uint32_t bar_final = bar0 + 192, bar_o_free = bar0 + 208;
-    constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA lane + two softmax warpgroups + correction warpgroup
+    const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144, bar_pv = bar0 + 160;
+    const uint32_t bar_final = bar0 + 176, bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
+    constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA warp + two softmax warpgroups + epilogue warpgroup
 
     if (tid == 0) {
         abort_flag = 0;
@@ -165,11 +181,11 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
             mbar_init(bar_q_full + 8 * i, 1);
             mbar_init(bar_q_free + 8 * i, 1);
             mbar_init(bar_s_full + 8 * i, 1);
-            mbar_init(bar_alpha + 8 * i, kTile);
-            mbar_init(bar_po + 8 * i, 2 * kTile);
+            mbar_init(bar_po + 8 * i, kTile);
             mbar_init(bar_pv + 8 * i, 1);
             mbar_init(bar_final + 8 * i, kTile);
             mbar_init(bar_o_free + 8 * i, kTile);
+            mbar_init(bar_o_done + 8 * i, 1);
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(bar_full + 8 * i, 1);
@@ -202,15 +218,10 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         mbar_arrive(bar_item_free + 8 * (k & 1));
         return w;
     };
-    // key tile j of an item: first the shared range [0, a_end), then the own range from b_start
-    auto tile_start = [&](const WsItem& it, int j) { return j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile; };
-    auto tile_valid = [&](const WsItem& it, const WsSlot& s, int j) {
-        return j < it.na ? min(kTile, it.a_end - j * kTile) : min(kTile, s.b_end - (it.b_start + (j - it.na) * kTile));
-    };
 
-    // register budget per warpgroup: 2 x 192 (softmax) + 80 (correction) + 48 (TMA/MMA) = 512 x 128
+    // register budget per warpgroup: 2 x 192 (softmax) + 64 (epilogue) + 64 (TMA/MMA) = 512 x 128
     if (warp >= 12) {
-        reg_dealloc<48>();
+        reg_dealloc<64>();
       if (warp == 13) {
         // ------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
@@ -238,7 +249,7 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                     ++q_loads[x];
                 }
                 for (int j = 0; j < nt_max; ++j) {
-                    const int j0 = tile_start(it, j);
+                    const int j0 = j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile;
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const int slot = ring_idx % kRing, use = ring_idx / kRing;
@@ -254,83 +265,119 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         }
       } else if (warp == 12) {
         // ------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            int ring_base = 0;        // ring position of this item's K(0)
-            int cnt[2] = {0, 0};      // tiles issued per slot so far (phase of s_full / po / pv)
-            int q_uses[2] = {0, 0};   // items in which the slot was active so far
-            for (int k = 0;; ++k) {
-                const int w = next_item(k);
-                if (w < 0) break;
-                WsItem it;
-                decode_ws_item(p, w, it);
-                const int nt0 = it.s[0].nt, nt1 = it.s[1].nt;
-                const int nt_max = max(nt0, nt1);
-                auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
-                auto wait_full = [&](int idx) {
-                    const int g = ring_base + idx;
-                    wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWsWaitFull);
-                };
-                auto commit_empty = [&](int idx) { mma_commit(bar_empty + 8 * ((ring_base + idx) % kRing)); };
-                auto issue_qk = [&](int x, int j) {
-                    const int n_mma = (tile_valid(it, it.s[x], j) + 15) & ~15;
-                    const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
-                    const uint32_t sq = smem_base + (x ? L::kQ1 : L::kQ0), sk = ring_addr(2 * j);
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (ks / 4) * L::kPanelBytes + (ks % 4) * 32;
-                        mma_ss(tmem_base + x * 128, make_smem_desc_sw128(sq + off, 16, 1024),
-                               make_smem_desc_sw128(sk + off, 16, 1024), idesc, ks > 0);
-                    }
-                    mma_commit(bar_s_full + 8 * x);
-                    if (j == it.s[x].nt - 1) mma_commit(bar_q_free + 8 * x);  // last use of this Q tile
-                };
-                auto issue_pv = [&](int x, int j) {
-                    wait(bar_po + 8 * x, (cnt[x] + j) & 1, kWsWaitPO);
-                    // the previous item's output must have left TMEM before O is overwritten
-                    if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWsWaitOFree);
-                    tc_fence_after_sync();
-                    const int ksteps = (tile_valid(it, it.s[x], j) + 15) >> 4;
-                    const uint32_t idesc = make_idesc_bf16(kTile, D, true);
-                    const uint32_t sv = ring_addr(2 * j + 1);
-                    for (int ks = 0; ks < ksteps; ++ks)
-                        mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + ks * 8,
-                               make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc, (j > 0) || (ks > 0));
-                    mma_commit(bar_pv + 8 * x);
-                };
-#pragma unroll
-                for (int x = 0; x < 2; ++x)
-                    if (it.s[x].nt > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWsWaitQ);
+        // All 32 lanes run this loop with warp-uniform values (descriptors and addresses stay in
+        // uniform registers); the MMA and commit instructions themselves go out from one elected lane.
+        int ring_base = 0;        // ring position of this item's K(0)
+        int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po / pv)
+        int q_uses[2] = {0, 0};   // items in which the slot was active so far
+        PROF_DECL(8)
+        for (int k = 0;; ++k) {
+            PROF_LAP(5)
+            // every lane reads the item, one lane releases the queue slot
+            wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWsWaitItem);
+            const int w = s_item[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_item_free + 8 * (k & 1));
+            PROF_LAP(0)
+            if (w < 0) break;
+            WsItem it;
+            decode_ws_item(p, w, it);
+            const int nt[2] = {it.s[0].nt, it.s[1].nt};
+            const int nt_max = max(nt[0], nt[1]);
+            // keys in the last tile of the shared range and of each slot's own range (every other
+            // tile is full)
+            const int na = it.na;
+            const int a_last = it.a_end - (na - 1) * kTile;
+            const int b_last[2] = {it.s[0].b_end - it.b_start - (nt[0] - na - 1) * kTile,
+                                   it.s[1].b_end - it.b_start - (nt[1] - na - 1) * kTile};
+            auto valid_of = [&](int x, int j) { return (j == na - 1) ? a_last : (j == nt[x] - 1) ? b_last[x] : kTile; };
+            auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
+            auto wait_full = [&](int idx) {
+                const int g = ring_base + idx;
+                PROF_LAP(5)
+                wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWsWaitFull);
+                PROF_LAP(2)
+            };
+            auto commit_empty = [&](int idx) { mma_commit_elect(bar_empty + 8 * ((ring_base + idx) % kRing)); };
+            // S_x = Q_x K(j)^T
+            auto issue_qk = [&](int x, int j) {
+                const int n_mma = (valid_of(x, j) + 15) & ~15;
+                const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
+                PROF_LAP(5)
+                mma_ss_batch<D / 16>(tmem_base + x * 128, desc_lo(smem_base + (x ? L::kQ1 : L::kQ0), 16),
+                                     desc_lo(ring_addr(2 * j), 16), idesc);
+                PROF_LAP(6)
+                mma_commit_elect(bar_s_full + 8 * x);
+                if (j == nt[x] - 1) mma_commit_elect(bar_q_free + 8 * x);  // last use of this Q tile
+                PROF_LAP(7)
+            };
+            // O_x += P_x V(j)
+            auto issue_pv = [&](int x, int j) {
+                PROF_LAP(5)
+                wait(bar_po + 8 * x, (cnt[x] + j) & 1, kWsWaitPO);
+                PROF_LAP(3)
+                // the previous item's output must have left TMEM before O is overwritten
+                if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWsWaitOFree);
+                PROF_LAP(4)
                 tc_fence_after_sync();
-                for (int j = 0; j <= nt_max; ++j) {
-                    if (j < nt_max) {
-                        wait_full(2 * j);
-                        tc_fence_after_sync();
-                        if (j < nt0) issue_qk(0, j);
-                    }
-                    if (j > 0) {
-                        if (j - 1 < nt1) {
-                            wait_full(2 * (j - 1) + 1);
-                            issue_pv(1, j - 1);
-                        }
-                        commit_empty(2 * (j - 1) + 1);  // V(j-1) consumed
-                    }
-                    if (j < nt_max) {
-                        if (j < nt1) issue_qk(1, j);
-                        commit_empty(2 * j);  // K(j) consumed
-                        if (j < nt0) {
-                            wait_full(2 * j + 1);
-                            issue_pv(0, j);
-                        }
-                    }
+                const int nvalid = valid_of(x, j);
+                const uint32_t idesc = make_idesc_bf16(kTile, D, true);
+                const uint32_t sv = ring_addr(2 * j + 1);
+                const uint32_t d_tmem = tmem_base + 256 + x * 128, a_tmem = tmem_base + x * 128;
+                PROF_LAP(5)
+                if (nvalid == kTile) {
+                    mma_ts_batch8(d_tmem, a_tmem, desc_lo(sv, L::kPanelBytes), idesc, j > 0);
+                } else {
+                    const int ksteps = (nvalid + 15) >> 4;
+                    for (int ks = 0; ks < ksteps; ++ks)
+                        mma_ts_elect(d_tmem, a_tmem + ks * 8, make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc,
+                                     (j > 0) || (ks > 0));
                 }
-                ring_base += 2 * nt_max;
+                PROF_LAP(1)
+                // pv: read by the softmax for its rare in-place rescale (one phase per tile);
+                // o_done: the item's accumulator is complete (one phase per item, for the epilogue)
+                mma_commit_elect(bar_pv + 8 * x);
+                if (j == nt[x] - 1) mma_commit_elect(bar_o_done + 8 * x);
+                PROF_LAP(7)
+            };
+            PROF_LAP(5)
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    cnt[x] += it.s[x].nt;
-                    if (it.s[x].nt > 0) ++q_uses[x];
+            for (int x = 0; x < 2; ++x)
+                if (nt[x] > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWsWaitQ);
+            PROF_LAP(4)
+            tc_fence_after_sync();
+            // order on the tensor pipe: QK0(j) PV1(j-1) QK1(j) PV0(j): while one query tile is in its
+            // softmax the other one's MMAs run
+            for (int j = 0; j <= nt_max; ++j) {
+                if (j < nt_max) {
+                    wait_full(2 * j);
+                    tc_fence_after_sync();
+                    if (j < nt[0]) issue_qk(0, j);
+                }
+                if (j > 0) {
+                    if (j - 1 < nt[1]) {
+                        wait_full(2 * (j - 1) + 1);
+                        issue_pv(1, j - 1);
+                    }
+                    commit_empty(2 * (j - 1) + 1);  // V(j-1) consumed
+                }
+                if (j < nt_max) {
+                    if (j < nt[1]) issue_qk(1, j);
+                    commit_empty(2 * j);  // K(j) consumed
+                    if (j < nt[0]) {
+                        wait_full(2 * j + 1);
+                        issue_pv(0, j);
+                    }
                 }
             }
+            ring_base += 2 * nt_max;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                cnt[x] += nt[x];
+                if (nt[x] > 0) ++q_uses[x];
+            }
         }
+        if (lane == 0) { PROF_DUMP(0, 8) }
       }
     } else if (warp < 8) {
         // ------------------------------------------------------------- softmax of slot x
@@ -339,38 +386,50 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + x * 128 + lane_off;
-        int cnt = 0;   // tiles of this slot processed so far (phase of s_full)
+        const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
+        const uint32_t my_s_full = bar_s_full + 8 * x, my_po = bar_po + 8 * x, my_pv = bar_pv + 8 * x;
+        int cnt = 0;   // tiles of this slot processed so far (phase of s_full / pv)
         int uses = 0;  // items in which this slot was active so far
+        PROF_DECL(8)
         for (int k = 0;; ++k) {
+            PROF_LAP(7)
             const int w = next_item(k);
+            PROF_LAP(0)
             if (w < 0) break;
             WsItem it;
             decode_ws_item(p, w, it);
-            const WsSlot& s = it.s[x];
-            if (s.nt == 0) continue;
-            const int my_limit = s.limit0 + row / it.row_div;
+            // this slot's scalars, in registers
+            const int nt = x ? it.s[1].nt : it.s[0].nt;
+            if (nt == 0) continue;
+            const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
+            const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
+            const int na = it.na, a_end = it.a_end, b_start = it.b_start;
+            const int my_limit = limit0 + row / it.row_div;
             float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
             float l_run = 0.f;
-            for (int j = 0; j < s.nt; ++j, ++cnt) {
-                const int j0 = tile_start(it, j);
-                const int nvalid = tile_valid(it, s, j);
-                const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > s.limit0);
-                const int max_col = need_mask ? min(nvalid, my_limit - j0 + 1) : kTile;
-                wait(bar_s_full + 8 * x, cnt & 1, kWsWaitS);
+            for (int j = 0; j < nt; ++j, ++cnt) {
+                const int j0 = j < na ? j * kTile : b_start + (j - na) * kTile;
+                const int nvalid = min(kTile, (j < na ? a_end : b_end) - j0);
+                const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > limit0);
+                PROF_LAP(7)
+                wait(my_s_full, cnt & 1, kWsWaitS);
+                PROF_LAP(1)
                 tc_fence_after_sync();
                 // all 128 scores of the row in registers: one round trip to TMEM
-                uint32_t r[128];
+                uint32_t r[kTile];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
                 tmem_wait_ld();
+                PROF_LAP(2)
                 if (need_mask) {
+                    const int max_col = min(nvalid, my_limit - j0 + 1);
 #pragma unroll
-                    for (int i = 0; i < 128; ++i)
+                    for (int i = 0; i < kTile; ++i)
                         if (i >= max_col) r[i] = 0xff800000u;  // -inf
                 }
                 float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int i = 0; i < 128; i += 8) {
+                for (int i = 0; i < kTile; i += 8) {
 #pragma unroll
                     for (int a = 0; a < 4; ++a)
                         mx[a] = fmax3(mx[a], __uint_as_float(r[i + 2 * a]), __uint_as_float(r[i + 2 * a + 1]));
@@ -382,10 +441,23 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                     alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
                     m_ref = m_new;
                 }
-                if (j > 0) {
-                    s_alpha[x][row] = alpha;
-                    mbar_arrive(bar_alpha + 8 * x);
+                PROF_LAP(3)
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    // rare: rescale this row of the O accumulator in place, once PV(j-1) has landed.
+                    // (S(j) is complete, so PV(j-2) is too: the wait is at most one phase behind.)
+                    wait(my_pv, (cnt - 1) & 1, kWsWaitPV);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
                 }
+                PROF_LAP(4)
                 const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
                 // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot)
                 float sm[4] = {0.f, 0.f, 0.f, 0.f};
@@ -402,11 +474,11 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                     tmem_st16(tS + c * 16, pk);
                 }
                 const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
+                PROF_LAP(5)
                 tmem_wait_st();
+                PROF_LAP(6)
                 tc_fence_before_sync();
-                // the first tile of an item has no O to correct: this thread also arrives for its
-                // correction partner, so the epilogue of the previous item is not on the MMA's path
-                mbar_arrive_n(bar_po + 8 * x, j == 0 ? 2 : 1);
+                mbar_arrive(my_po);
                 l_run = l_run * alpha + sum;
             }
             s_final_l[uses & 1][x][row] = l_run;
@@ -414,45 +486,18 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
             mbar_arrive(bar_final + 8 * x);
             ++uses;
         }
+        if (tid == 0 || tid == 128) { PROF_DUMP(8 + 8 * x, 8) }
     } else {
-        // ------------------------------------------------------------- correction + epilogue
-        reg_dealloc<80>();
+        // ------------------------------------------------------------- epilogue
+        reg_dealloc<64>();
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        int cnt[2] = {0, 0};    // tiles per slot so far (phase of pv; alpha runs one behind per item)
-        int acnt[2] = {0, 0};   // alpha phases per slot so far (tiles with j > 0)
-        int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_free)
+        int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_done / o_free)
         for (int k = 0;; ++k) {
             const int w = next_item(k);
             if (w < 0) break;
             WsItem it;
             decode_ws_item(p, w, it);
-            const int nt_max = max(it.s[0].nt, it.s[1].nt);
-            for (int j = 1; j < nt_max; ++j) {
-#pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    if (j >= it.s[x].nt) continue;
-                    wait(bar_alpha + 8 * x, (acnt[x] + j - 1) & 1, kWsWaitAlpha);
-                    const float alpha = s_alpha[x][row];
-                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
-                        wait(bar_pv + 8 * x, (cnt[x] + j - 1) & 1, kWsWaitPV);
-                        tc_fence_after_sync();
-                        const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
-#pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                            tmem_st32(tO + c * 32, o);
-                        }
-                        tmem_wait_st();
-                    }
-                    tc_fence_before_sync();
-                    mbar_arrive(bar_po + 8 * x);
-                }
-            }
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 const WsSlot& s = it.s[x];
@@ -471,9 +516,9 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                     continue;
                 }
                 wait(bar_final + 8 * x, uses[x] & 1, kWsWaitFinal);
-                wait(bar_pv + 8 * x, (cnt[x] + s.nt - 1) & 1, kWsWaitPV);
-                tc_fence_after_sync();
                 const float l = s_final_l[uses[x] & 1][x][row], m = s_final_m[uses[x] & 1][x][row];
+                wait(bar_o_done + 8 * x, uses[x] & 1, kWsWaitPV);
+                tc_fence_after_sync();
                 const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
                 const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
                 const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
@@ -517,14 +562,8 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                 }
             }
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const int nt = it.s[x].nt;
-                cnt[x] += nt;
-                if (nt > 0) {
-                    acnt[x] += nt - 1;
-                    ++uses[x];
-                }
-            }
+            for (int x = 0; x < 2; ++x)
+                if (it.s[x].nt > 0) ++uses[x];
         }
     }
     tc_fence_before_sync();

@@ -128,6 +128,21 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Warp-collective forms: every lane calls them, one elected lane issues.
+__device__ __forceinline__ void mma_commit_elect(uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_elect(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(static_cast<uint32_t>(accumulate)));
+}
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -186,6 +201,76 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_
     d |= 1ull << 46;
     d |= 2ull << 61;
     return d;
+}
+
+// ---- batched MMA issue.  The issuing thread is latency-bound on its own instruction stream,
+// so a whole k-loop goes out as one asm block: descriptors are a constant high word plus a
+// low word (address >> 4 | leading byte offset >> 4 << 16) that only needs an add per step.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024 B, version 1, 128-byte swizzle
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+
+// These are called by ALL lanes of the issuing warp with warp-uniform operands (so the
+// operands live in uniform registers); one elected lane issues.
+#define PEVLM_MMA_SS_STEP(OFF, PRED)                                              \
+    "add.u32 ta, %1, " #OFF ";\n\tadd.u32 tb, %2, " #OFF ";\n\t"                  \
+    "mov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"                          \
+    "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " PRED ";\n\t"
+
+// D[tmem] = A[smem] * B[smem]^T over head_dim = 16 * KSTEPS; A and B are K-major, 128-byte
+// swizzled tiles whose 64-element column panels are 16 KB apart.  The first step overwrites D.
+template <int KSTEPS>
+__device__ __forceinline__ void mma_ss_batch(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+    static_assert(KSTEPS == 4 || KSTEPS == 8, "head_dim 64 or 128");
+    if constexpr (KSTEPS == 8) {
+        asm volatile(
+            "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+            PEVLM_MMA_SS_STEP(0, "p0") PEVLM_MMA_SS_STEP(2, "p1") PEVLM_MMA_SS_STEP(4, "p1") PEVLM_MMA_SS_STEP(6, "p1")
+            PEVLM_MMA_SS_STEP(1024, "p1") PEVLM_MMA_SS_STEP(1026, "p1") PEVLM_MMA_SS_STEP(1028, "p1") PEVLM_MMA_SS_STEP(1030, "p1")
+            "}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc));
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+            PEVLM_MMA_SS_STEP(0, "p0") PEVLM_MMA_SS_STEP(2, "p1") PEVLM_MMA_SS_STEP(4, "p1") PEVLM_MMA_SS_STEP(6, "p1")
+            "}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc));
+    }
+}
+
+#define PEVLM_MMA_TS_STEP(AOFF, BOFF, PRED)                                       \
+    "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                \
+    "mov.b64 db, {tb, %3};\n\t"                                                   \
+    "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %4, " PRED ";\n\t"
+
+// D[tmem] (+)= A[tmem] * B[smem] over 64 keys (four steps of 16): A = bf16 probabilities, 8
+// TMEM columns per step; B = V rows (MN-major, 16 keys = 2048 bytes per step).  The first step
+// accumulates iff accumulate_first != 0.
+__device__ __forceinline__ void mma_ts_batch4(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t accumulate_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b32 ta, tb;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        PEVLM_MMA_TS_STEP(0, 0, "p0") PEVLM_MMA_TS_STEP(8, 128, "p1") PEVLM_MMA_TS_STEP(16, 256, "p1")
+        PEVLM_MMA_TS_STEP(24, 384, "p1")
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate_first));
+}
+
+// Same over 128 keys (eight steps).
+__device__ __forceinline__ void mma_ts_batch8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t accumulate_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b32 ta, tb;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        PEVLM_MMA_TS_STEP(0, 0, "p0") PEVLM_MMA_TS_STEP(8, 128, "p1") PEVLM_MMA_TS_STEP(16, 256, "p1")
+        PEVLM_MMA_TS_STEP(24, 384, "p1") PEVLM_MMA_TS_STEP(32, 512, "p1") PEVLM_MMA_TS_STEP(40, 640, "p1")
+        PEVLM_MMA_TS_STEP(48, 768, "p1") PEVLM_MMA_TS_STEP(56, 896, "p1")
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate_first));
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {

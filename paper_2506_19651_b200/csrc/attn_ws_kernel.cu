@@ -219,9 +219,9 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
         return w;
     };
 
-    // register budget per warpgroup: 2 x 192 (softmax) + 64 (epilogue) + 64 (TMA/MMA) = 512 x 128
+    // register budget per warpgroup: 2 x 200 (softmax) + 64 (epilogue) + 48 (TMA/MMA) = 512 x 128
     if (warp >= 12) {
-        reg_dealloc<64>();
+        reg_dealloc<48>();
       if (warp == 13) {
         // ------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
@@ -381,7 +381,7 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
       }
     } else if (warp < 8) {
         // ------------------------------------------------------------- softmax of slot x
-        reg_alloc<192>();
+        reg_alloc<200>();
         const int x = warp >> 2;
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -459,21 +459,33 @@ attn_ws_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUt
                 }
                 PROF_LAP(4)
                 const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
-                // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot)
-                float sm[4] = {0.f, 0.f, 0.f, 0.f};
+                // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot);
+                // scale-and-shift and the row sum run as packed fp32 pairs
+                const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+                const uint64_t shift2 = pack_f32x2(neg_ms, neg_ms);
+                uint64_t sm2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i]), p.scale_log2, neg_ms));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 32 + 2 * i + 1]), p.scale_log2, neg_ms));
-                        sm[i & 3] += p0 + p1;
+                        const uint64_t t2 = fma_f32x2(pack_f32x2(__uint_as_float(r[c * 32 + 2 * i]),
+                                                                 __uint_as_float(r[c * 32 + 2 * i + 1])), scale2, shift2);
+                        float t0, t1;
+                        unpack_f32x2(t2, t0, t1);
+                        const float p0 = fast_exp2(t0), p1 = fast_exp2(t1);
+                        sm2[i & 3] = add_f32x2(sm2[i & 3], pack_f32x2(p0, p1));
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(tS + c * 16, pk);
                 }
-                const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
+                float sum;
+                {
+                    float a0, a1, b0, b1;
+                    unpack_f32x2(add_f32x2(sm2[0], sm2[1]), a0, a1);
+                    unpack_f32x2(add_f32x2(sm2[2], sm2[3]), b0, b1);
+                    sum = (a0 + a1) + (b0 + b1);
+                }
                 PROF_LAP(5)
                 tmem_wait_st();
                 PROF_LAP(6)

@@ -3,7 +3,6 @@
 // except pevlm_read_status.
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 
 #include "internal.h"
@@ -87,12 +86,6 @@ static int make_tmap(CUtensorMap* m, const void* base, int64_t tokens, int heads
         return PEVLM_ECUDA;
     }
     return PEVLM_OK;
-}
-
-// Development switch: PEVLM_ATTN_SIMPLE=1 selects the single-tile, non-specialised kernel.
-static bool use_simple_kernel() {
-    const char* e = getenv("PEVLM_ATTN_SIMPLE");
-    return e && e[0] == '1';
 }
 
 static float resolve_scale(const pevlm_shape_t* s) {
@@ -250,16 +243,10 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
     p.Hq = s->num_q_heads; p.Hkv = s->num_kv_heads; p.G = p.Hq / p.Hkv;
     p.tiles_sink = (p.S + kTile - 1) / kTile;
     p.tiles_block = p.N > 0 ? (p.B + kTile - 1) / kTile : 0;
-    const bool simple = use_simple_kernel();
-    if (simple) {
-        p.items_block = p.N * p.tiles_block * p.Hq;
-        p.n_items = p.items_block + p.tiles_sink * p.Hq;
-    } else {
-        p.pairs_block = (p.G * p.tiles_block + 1) / 2;
-        p.pairs_sink = (p.G * p.tiles_sink + 1) / 2;
-        p.items_block = p.N * p.Hkv * p.pairs_block;
-        p.n_items = p.items_block + p.Hkv * p.pairs_sink;
-    }
+    p.pairs_block = (p.G * p.tiles_block + 1) / 2;
+    p.pairs_sink = (p.G * p.tiles_sink + 1) / 2;
+    p.items_block = p.N * p.Hkv * p.pairs_block;
+    p.n_items = p.items_block + p.Hkv * p.pairs_sink;
     p.q_box_rows = kTile;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
@@ -276,7 +263,7 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
             e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
             if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
         }
-        e = simple ? launch_attn(p, d, tq, tk, tv, st) : launch_attn_ws(p, d, tq, tk, tv, st);
+        e = launch_attn(p, d, tq, tk, tv, st);
         if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
     }
     return PEVLM_OK;
@@ -314,8 +301,7 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
     p.n_splits = qp.n_splits;
     p.tiles_per_split = qp.tiles_per_split;
     p.q_box_rows = p.G * p.tok_per_tile;
-    const bool simple = use_simple_kernel();
-    p.n_items = p.Hkv * (simple ? p.q_tiles : (p.q_tiles + 1) / 2) * p.n_splits;
+    p.n_items = p.Hkv * ((p.q_tiles + 1) / 2) * p.n_splits;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
     p.hdr = static_cast<WorkspaceHeader*>(workspace);
@@ -334,7 +320,7 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
         if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        e = simple ? launch_attn(p, d, tq, tk, tv, st) : launch_attn_ws(p, d, tq, tk, tv, st);
+        e = launch_attn(p, d, tq, tk, tv, st);
         if (e != cudaSuccess) return cuda_fail(e, "question attention launch");
         MergeParams m;
         m.Q = p.Q; m.Hq = p.Hq; m.d = d; m.n_splits = p.n_splits;

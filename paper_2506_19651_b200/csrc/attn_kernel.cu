@@ -1,422 +1,610 @@
-// Block-masked flash attention for sm_100a (Eq. 1 under the masks of Eq. 3-5).
+// Warp-specialised block-masked flash attention for sm_100a (Eq. 1 under the masks of Eq. 3-5).
 //
-// One CTA computes one query tile of 128 rows against the key tiles that tile can see:
-//   prefill rows of context block i : the sink's tiles, then block i's tiles up to the diagonal
-//   sink rows / full-causal rows    : tiles up to the diagonal
-//   question rows (split over keys) : a contiguous slice of the cache's tiles
-// Key/value tiles arrive by TMA (128-byte swizzle) into a two-stage ring; S = Q K^T and
-// O += P V run on the tensor cores (tcgen05.mma, accumulators in TMEM, P fed back from TMEM
-// as the A operand); the online softmax runs in fp32 with one thread per query row.
+// One CTA owns TWO query tiles of 128 rows that share a kv head and a key-tile list (two q
+// heads of one GQA group at the same block position, or two neighbouring positions), so every
+// K/V tile staged in shared memory feeds both.  Roles (16 warps):
+//   warps 0-3   softmax of query tile 0: one thread per row; the 128 scores of a key tile are
+//               read from TMEM once, running max/sum kept in fp32, probabilities written back
+//               over the scores as bf16; the rare rescale of the O accumulator (the reference
+//               maximum moves only when a row's maximum grows by more than 2^8) is done in
+//               place by the same threads
+//   warps 4-7   softmax of query tile 1
+//   warps 8-11  epilogue: normalised output and LSE of a finished item, TMEM -> global
+//   warp 12     issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
+//               O += P V (P from TMEM, V from shared memory), ping-ponging between the two
+//               query tiles so one is in the tensor cores while the other is in its softmax
+//   warp 13     work scheduler and TMA producer: takes the next work item from a global
+//               counter, publishes it to the other roles, loads its two Q tiles, then streams
+//               K/V tiles through a 4-slot ring that runs on across items
+// The kernel is persistent (one CTA per SM): while the correction warps write out item k, the
+// producer, the MMA warp and the softmax warps already work on item k+1.
+// TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
+// Every wait is bounded; an expired wait records PEVLM_ETIMEOUT and the CTA still runs to its
+// normal end (waits become short), so TMEM is always released.
 #include "internal.h"
 #include "ptx.cuh"
 
 namespace pevlm {
 
-constexpr int kAttnThreads = 128;
-constexpr int kStages = 2;
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemS = 0;    // 128 fp32 columns: scores
-constexpr uint32_t kTmemP = 128;  // 64 columns: probabilities, two bf16 per column
-constexpr uint32_t kTmemO = 256;  // d fp32 columns: output accumulator
+constexpr int kAttnThreads = 512;
+constexpr int kRing = 4;
+constexpr float kRescaleThresholdLog2 = 8.0f;  // rescale O only when the row maximum grew by > 2^8
 
-// wait identifiers recorded in the workspace header when a bounded wait expires
-enum WaitId : int { kWaitQ = 1, kWaitK = 2, kWaitV = 3, kWaitS = 4, kWaitO = 5 };
+enum WaitId : int {
+    kWaitQ = 11, kWaitFull = 12, kWaitEmpty = 13, kWaitS = 14, kWaitAlpha = 15,
+    kWaitPO = 16, kWaitPV = 17, kWaitFinal = 18, kWaitItem = 19, kWaitItemFree = 20,
+    kWaitQFree = 21, kWaitOFree = 22
+};
+
+// Optional in-kernel cycle accounting (compile with -DPEVLM_PROFILE): CTA 0 accumulates the
+// cycles its MMA thread and one softmax thread spend in each wait / phase and leaves them in
+// the padding of the workspace header.
+#ifdef PEVLM_PROFILE
+#define PROF_DECL(n) long long prof_acc[n] = {}; long long prof_t = clock64();
+#define PROF_LAP(i) { const long long prof_now = clock64(); prof_acc[i] += prof_now - prof_t; prof_t = prof_now; }
+#define PROF_DUMP(base, n) if (blockIdx.x == 0) { for (int prof_i = 0; prof_i < (n); ++prof_i) p.hdr->pad[(base) + prof_i] = static_cast<int32_t>(prof_acc[prof_i] >> 4); }
+#else
+#define PROF_DECL(n)
+#define PROF_LAP(i)
+#define PROF_DUMP(base, n)
+#endif
 
 template <int D>
-struct SmemLayout {
-    static constexpr int kHalves = D / 64;                 // 64-element (128-byte) column panels
-    static constexpr int kPanelBytes = kTile * 128;        // 128 rows x 128 bytes
-    static constexpr int kTileBytes = kHalves * kPanelBytes;
-    static constexpr int kQ = 0;
-    static constexpr int kK = kTileBytes;
-    static constexpr int kV = kK + kStages * kTileBytes;
-    static constexpr int kTotal = kV + kStages * kTileBytes;
+struct AttnSmem {
+    static constexpr int kPanels = D / 64;
+    static constexpr int kPanelBytes = kTile * 128;
+    static constexpr int kTileBytes = kPanels * kPanelBytes;
+    static constexpr int kQ0 = 0;
+    static constexpr int kQ1 = kTileBytes;
+    static constexpr int kRing0 = 2 * kTileBytes;
+    static constexpr int kTotal = kRing0 + kRing * kTileBytes;
 };
 
 size_t attn_smem_bytes(int head_dim) {
-    return 1024 + (head_dim == 128 ? SmemLayout<128>::kTotal : SmemLayout<64>::kTotal);
+    return 1024 + (head_dim == 128 ? AttnSmem<128>::kTotal : AttnSmem<64>::kTotal);
 }
 
-struct Item {
-    int q_tok0;      // first token of the query tile (row of the q tensor)
-    int q_head0;     // first head of the TMA box
-    int kv_head;
-    int rows_valid;  // rows of the tile that exist
-    int row_div;     // rows per token (1 prefill, G question)
-    int limit0;      // key index visible limit of row r: limit0 + r / row_div (inclusive)
-    int a_start, a_end;  // first key range  [a_start, a_end)
-    int b_start, b_end;  // second key range [b_start, b_end)
-    int split;       // question mode
+struct QSlot {
+    int valid;
+    int q_tok0, q_head0, rows_valid, limit0, b_end, nt;
+};
+struct WorkItem {
+    int kv_head, row_div, a_end, b_start, na, split;
+    QSlot s[2];
 };
 
-__device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+__device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
 
-__device__ __forceinline__ Item decode_item(const AttnParams& p, int w) {
-    Item it;
+__device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem& it) {
     it.split = 0;
     if (p.mode == 0) {
         it.row_div = 1;
+        int seg_start, seg_len, tiles, pi, g;
         if (w < p.items_block) {
-            // context-block rows, heaviest query tiles (largest index in the block) first
-            const int per_qt = p.N * p.Hq;
-            const int qt = p.tiles_block - 1 - w / per_qt;
-            const int rem = w % per_qt;
-            const int blk = rem / p.Hq;
-            const int h = rem % p.Hq;
-            const int blk_start = p.S + blk * p.B;
-            it.q_tok0 = blk_start + qt * kTile;
-            it.q_head0 = h;
-            it.kv_head = h / p.G;
-            it.rows_valid = min(kTile, p.B - qt * kTile);
-            it.limit0 = it.q_tok0;
-            it.a_start = 0;
+            const int combo = w / p.pairs_block;
+            pi = w % p.pairs_block;
+            const int blk = combo / p.Hkv;
+            g = combo % p.Hkv;
+            seg_start = p.S + blk * p.B;
+            seg_len = p.B;
+            tiles = p.tiles_block;
             it.a_end = p.S;
-            it.b_start = blk_start;
-            it.b_end = min(it.q_tok0 + kTile, blk_start + p.B);
         } else {
             const int w2 = w - p.items_block;
-            const int qt = p.tiles_sink - 1 - w2 / p.Hq;
-            const int h = w2 % p.Hq;
-            it.q_tok0 = qt * kTile;
-            it.q_head0 = h;
-            it.kv_head = h / p.G;
-            it.rows_valid = min(kTile, p.S - qt * kTile);
-            it.limit0 = it.q_tok0;
-            it.a_start = 0;
+            g = w2 / p.pairs_sink;
+            pi = w2 % p.pairs_sink;
+            seg_start = 0;
+            seg_len = p.S;
+            tiles = p.tiles_sink;
             it.a_end = 0;
-            it.b_start = 0;
-            it.b_end = min(it.q_tok0 + kTile, p.S);
+        }
+        it.kv_head = g;
+        it.b_start = seg_start;
+        it.na = cdiv(it.a_end, kTile);
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int e = 2 * pi + x;
+            QSlot& s = it.s[x];
+            s.valid = e < p.G * tiles;
+            const int qt = tiles - 1 - e / p.G;  // heaviest query tiles first
+            s.q_tok0 = seg_start + qt * kTile;
+            s.q_head0 = g * p.G + e % p.G;
+            s.rows_valid = min(kTile, seg_len - qt * kTile);
+            s.limit0 = s.q_tok0;
+            s.b_end = min(s.q_tok0 + kTile, seg_start + seg_len);
+            s.nt = s.valid ? it.na + cdiv(s.b_end - it.b_start, kTile) : 0;
         }
     } else {
         it.split = w % p.n_splits;
         const int rest = w / p.n_splits;
-        const int qt = rest % p.q_tiles;
-        const int g = rest / p.q_tiles;
-        const int tok0 = qt * p.tok_per_tile;
-        const int ntok = min(p.tok_per_tile, p.Q - tok0);
-        it.q_tok0 = tok0;
-        it.q_head0 = g * p.G;
+        const int q_pairs = cdiv(p.q_tiles, 2);
+        const int pi = rest % q_pairs;
+        const int g = rest / q_pairs;
         it.kv_head = g;
-        it.rows_valid = ntok * p.G;
         it.row_div = p.G;
-        it.limit0 = p.n_video + tok0;
-        const int kv_end = p.n_video + tok0 + ntok;  // keys beyond the last row's limit are never visible
-        it.a_start = 0;
         it.a_end = 0;
-        it.b_start = min(kv_end, it.split * p.tiles_per_split * kTile);
-        it.b_end = min(kv_end, (it.split + 1) * p.tiles_per_split * kTile);
+        it.na = 0;
+        const int split_lo = it.split * p.tiles_per_split * kTile;
+        const int split_hi = split_lo + p.tiles_per_split * kTile;
+        it.b_start = split_lo;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int qt = 2 * pi + x;
+            QSlot& s = it.s[x];
+            s.valid = qt < p.q_tiles;
+            const int tok0 = qt * p.tok_per_tile;
+            const int ntok = max(0, min(p.tok_per_tile, p.Q - tok0));
+            s.q_tok0 = tok0;
+            s.q_head0 = g * p.G;
+            s.rows_valid = ntok * p.G;
+            s.limit0 = p.n_video + tok0;
+            const int kv_end = p.n_video + tok0 + ntok;  // keys past the last row's limit are never visible
+            s.b_end = min(kv_end, split_hi);
+            s.nt = (s.valid && s.b_end > split_lo) ? cdiv(s.b_end - split_lo, kTile) : 0;
+        }
     }
-    return it;
 }
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap tmap_q,
-            const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
-    using L = SmemLayout<D>;
-    constexpr int NH = L::kHalves;
+               const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+    using L = AttnSmem<D>;
+    constexpr int NP = L::kPanels;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[3 + 2 * kStages];
+    // barrier map (uint64 each): [0,2) item_full [2,4) item_free [4,6) q_full [6,8) q_free
+    // [8,12) ring full [12,16) ring empty, then per slot x: [16,18) s_full [18,20) po [20,22) pv
+    // [22,24) final [24,26) o_free [26,28) o_done
+    __shared__ uint64_t bars[28];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int s_item[2];
+    __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a short
+    __shared__ float s_final_m[2][2][kTile];  // item while the previous item's epilogue is still running
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+    const int lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base + L::kQ;
-    const uint32_t sK = smem_base + L::kK;
-    const uint32_t sV = smem_base + L::kV;
-    const uint32_t bar_q = smem_u32(&bars[0]);
-    const uint32_t bar_s = smem_u32(&bars[1]);
-    const uint32_t bar_o = smem_u32(&bars[2]);
-    const uint32_t bar_k0 = smem_u32(&bars[3]);
-    const uint32_t bar_v0 = smem_u32(&bars[3 + kStages]);
-
-    // an earlier CTA of this launch gave up on a wait: do no work (decided once per CTA)
-    if (tid == 0) abort_flag = p.hdr->status;
-    __syncthreads();
-    if (abort_flag != 0) return;
-
-    const Item it = decode_item(p, blockIdx.x);
-    const int na = ceil_div(it.a_end - it.a_start, kTile);
-    const int nb = ceil_div(it.b_end - it.b_start, kTile);
-    const int nt = na + nb;
-
-    if (nt == 0) {
-        // question-mode split with no visible key: neutral partial (weight 0 in the merge)
-        if (p.mode == 1 && tid < it.rows_valid) {
-            const int tok = it.q_tok0 + tid / it.row_div;
-            const int head = it.q_head0 + tid % it.row_div;
-            const size_t row = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-            p.part_lse[row] = -INFINITY;
-            float4* dst = reinterpret_cast<float4*>(p.part_o + row * D);
-            for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        return;
-    }
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    const uint32_t bar_item_full = bar0, bar_item_free = bar0 + 16, bar_q_full = bar0 + 32, bar_q_free = bar0 + 48;
+    const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
+    const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144, bar_pv = bar0 + 160;
+    const uint32_t bar_final = bar0 + 176, bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
+    constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA warp + two softmax warpgroups + epilogue warpgroup
 
     if (tid == 0) {
-        for (int i = 0; i < 3 + 2 * kStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_item_full + 8 * i, 1);
+            mbar_init(bar_item_free + 8 * i, kItemConsumers);
+            mbar_init(bar_q_full + 8 * i, 1);
+            mbar_init(bar_q_free + 8 * i, 1);
+            mbar_init(bar_s_full + 8 * i, 1);
+            mbar_init(bar_po + 8 * i, kTile);
+            mbar_init(bar_pv + 8 * i, 1);
+            mbar_init(bar_final + 8 * i, kTile);
+            mbar_init(bar_o_free + 8 * i, kTile);
+            mbar_init(bar_o_done + 8 * i, 1);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tmap_q);
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
     }
-    if (warp == 0) {
+    if (warp == 12) {
         __syncwarp();
-        tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
-    const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
-    const uint32_t tS = tmem_base + kTmemS, tP = tmem_base + kTmemP, tO = tmem_base + kTmemO;
 
-    auto tile_start = [&](int i) { return i < na ? it.a_start + i * kTile : it.b_start + (i - na) * kTile; };
-    auto tile_valid = [&](int i) {
-        return i < na ? min(kTile, it.a_end - (it.a_start + i * kTile)) : min(kTile, it.b_end - (it.b_start + (i - na) * kTile));
-    };
-    auto issue_kv_loads = [&](int i) {
-        const int s = i % kStages;
-        const int j0 = tile_start(i);
-        mbar_arrive_expect_tx(bar_k0 + 8 * s, L::kTileBytes);
-        for (int h = 0; h < NH; ++h)
-            tma_load_3d(sK + s * L::kTileBytes + h * L::kPanelBytes, &tmap_k, h * 64, it.kv_head, j0, bar_k0 + 8 * s);
-        mbar_arrive_expect_tx(bar_v0 + 8 * s, L::kTileBytes);
-        for (int h = 0; h < NH; ++h)
-            tma_load_3d(sV + s * L::kTileBytes + h * L::kPanelBytes, &tmap_v, h * 64, it.kv_head, j0, bar_v0 + 8 * s);
-    };
-    auto issue_qk = [&](int i) {
-        const int s = i % kStages;
-        const int n_mma = (tile_valid(i) + 15) & ~15;
-        const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t off = (ks / 4) * L::kPanelBytes + (ks % 4) * 32;
-            const uint64_t a = make_smem_desc_sw128(sQ + off, 16, 1024);
-            const uint64_t b = make_smem_desc_sw128(sK + s * L::kTileBytes + off, 16, 1024);
-            mma_ss(tS, a, b, idesc, ks > 0);
-        }
-        mma_commit(bar_s);
-    };
-    auto issue_pv = [&](int i) {
-        const int s = i % kStages;
-        const int ksteps = (tile_valid(i) + 15) >> 4;
-        const uint32_t idesc = make_idesc_bf16(kTile, D, true);
-        for (int ks = 0; ks < ksteps; ++ks) {
-            // V tile is [key][d] with d contiguous: MN-major B operand; 16 keys = 2048 bytes
-            const uint64_t b = make_smem_desc_sw128(sV + s * L::kTileBytes + ks * 2048, L::kPanelBytes, 1024);
-            mma_ts(tO, tP + ks * 8, b, idesc, (i > 0) || (ks > 0));
-        }
-        mma_commit(bar_o);
-    };
     auto give_up = [&](int which) {
         if (atomicCAS(&p.hdr->status, 0, PEVLM_ETIMEOUT) == 0) p.hdr->detail = which * 1000000 + blockIdx.x;
     };
+    auto wait = [&](uint32_t bar, uint32_t parity, int which) {
+        if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
+    };
+    // consumer side of the item queue: k-th item of this CTA, -1 = no more work
+    auto next_item = [&](int k) {
+        wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
+        const int w = s_item[k & 1];
+        mbar_arrive(bar_item_free + 8 * (k & 1));
+        return w;
+    };
 
-    if (tid == 0) {
-        mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(NH * p.q_box_rows * 128));
-        for (int h = 0; h < NH; ++h)
-            tma_load_3d(sQ + h * L::kPanelBytes, &tmap_q, h * 64, it.q_head0, it.q_tok0, bar_q);
-        issue_kv_loads(0);
-        if (nt > 1) issue_kv_loads(1);
-    }
-    if (!mbar_wait(bar_q, 0, &abort_flag)) give_up(kWaitQ);
-    if (!mbar_wait(bar_k0, 0, &abort_flag)) give_up(kWaitK);
-    tc_fence_after_sync();
-    if (tid == 0) issue_qk(0);
-
-    const int my_limit = it.limit0 + tid / it.row_div;
-    float m_run = -INFINITY;  // running maximum of the raw scores
-    float l_run = 0.f;        // running sum of exp2((s - m) * scale_log2)
-
-    for (int i = 0; i < nt; ++i) {
-        const int s = i % kStages;
-        const int j0 = tile_start(i);
-        const int nvalid = tile_valid(i);
-        const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > it.limit0);
-
-        if (!mbar_wait(bar_s, i & 1, &abort_flag)) give_up(kWaitS);
-        tc_fence_after_sync();
-
-        uint32_t sr[4][32];
+    // register budget per warpgroup: 2 x 200 (softmax) + 64 (epilogue) + 48 (TMA/MMA) = 512 x 128
+    if (warp >= 12) {
+        reg_dealloc<48>();
+      if (warp == 13) {
+        // ------------------------------------------------------------- scheduler + TMA producer
+        if (lane == 0) {
+            int ring_idx = 0;          // K/V tiles loaded so far (ring position), runs on across items
+            int q_loads[2] = {0, 0};   // Q loads per slot so far
+            for (int k = 0;; ++k) {
+                int w = (k == 0) ? static_cast<int>(blockIdx.x)
+                                 : static_cast<int>(gridDim.x) + atomicAdd(&p.hdr->work_counter, 1);
+                if (w >= p.n_items || abort_flag != 0 || *reinterpret_cast<volatile int32_t*>(&p.hdr->status) != 0) w = -1;
+                if (k >= 2) wait(bar_item_free + 8 * (k & 1), ((k >> 1) - 1) & 1, kWaitItemFree);
+                s_item[k & 1] = w;
+                mbar_arrive(bar_item_full + 8 * (k & 1));
+                if (w < 0) break;
+                WorkItem it;
+                decode_item(p, w, it);
+                const int nt_max = max(it.s[0].nt, it.s[1].nt);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sr[c]);
-        tmem_wait_ld();
-
-        float m_tile = -INFINITY;
-        if (need_mask) {
-            const int max_col = min(nvalid, my_limit - j0 + 1);  // columns [0, max_col) are visible
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float v = (c * 32 + j < max_col) ? __uint_as_float(sr[c][j]) : -INFINITY;
-                    sr[c][j] = __float_as_uint(v);
-                    m_tile = fmaxf(m_tile, v);
+                for (int x = 0; x < 2; ++x) {
+                    if (it.s[x].nt == 0) continue;
+                    if (q_loads[x] > 0) wait(bar_q_free + 8 * x, (q_loads[x] - 1) & 1, kWaitQFree);
+                    mbar_arrive_expect_tx(bar_q_full + 8 * x, static_cast<uint32_t>(NP * p.q_box_rows * 128));
+                    for (int h = 0; h < NP; ++h)
+                        tma_load_3d(smem_base + (x ? L::kQ1 : L::kQ0) + h * L::kPanelBytes, &tmap_q, h * 64,
+                                    it.s[x].q_head0, it.s[x].q_tok0, bar_q_full + 8 * x);
+                    ++q_loads[x];
                 }
-        } else {
+                for (int j = 0; j < nt_max; ++j) {
+                    const int j0 = j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int j = 0; j < 32; ++j) m_tile = fmaxf(m_tile, __uint_as_float(sr[c][j]));
-        }
-        const float m_new = fmaxf(m_run, m_tile);
-        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = fast_exp2((m_run - m_safe) * p.scale_log2);  // m_run = -inf -> 0
-        const float neg_ms = -m_safe * p.scale_log2;
-
-        uint32_t pk[64];
-        float sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * j]), p.scale_log2, neg_ms));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * j + 1]), p.scale_log2, neg_ms));
-                sum += p0 + p1;
-                pk[c * 16 + j] = pack_bf16x2(p0, p1);
+                    for (int kv = 0; kv < 2; ++kv) {
+                        const int slot = ring_idx % kRing, use = ring_idx / kRing;
+                        if (use > 0) wait(bar_empty + 8 * slot, (use - 1) & 1, kWaitEmpty);
+                        mbar_arrive_expect_tx(bar_full + 8 * slot, L::kTileBytes);
+                        for (int h = 0; h < NP; ++h)
+                            tma_load_3d(smem_base + L::kRing0 + slot * L::kTileBytes + h * L::kPanelBytes,
+                                        kv ? &tmap_v : &tmap_k, h * 64, it.kv_head, j0, bar_full + 8 * slot);
+                        ++ring_idx;
+                    }
+                }
             }
-        l_run = l_run * alpha + sum;
-        m_run = m_new;
-
-        if (i > 0) {
-            // PV(i-1) must be complete before O is rescaled, P overwritten, or its stage refilled
-            if (!mbar_wait(bar_o, (i - 1) & 1, &abort_flag)) give_up(kWaitO);
+        }
+      } else if (warp == 12) {
+        // ------------------------------------------------------------- MMA issuer
+        // All 32 lanes run this loop with warp-uniform values (descriptors and addresses stay in
+        // uniform registers); the MMA and commit instructions themselves go out from one elected lane.
+        int ring_base = 0;        // ring position of this item's K(0)
+        int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po / pv)
+        int q_uses[2] = {0, 0};   // items in which the slot was active so far
+        PROF_DECL(8)
+        for (int k = 0;; ++k) {
+            PROF_LAP(5)
+            // every lane reads the item, one lane releases the queue slot
+            wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
+            const int w = s_item[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_item_free + 8 * (k & 1));
+            PROF_LAP(0)
+            if (w < 0) break;
+            WorkItem it;
+            decode_item(p, w, it);
+            const int nt[2] = {it.s[0].nt, it.s[1].nt};
+            const int nt_max = max(nt[0], nt[1]);
+            // keys in the last tile of the shared range and of each slot's own range (every other
+            // tile is full)
+            const int na = it.na;
+            const int a_last = it.a_end - (na - 1) * kTile;
+            const int b_last[2] = {it.s[0].b_end - it.b_start - (nt[0] - na - 1) * kTile,
+                                   it.s[1].b_end - it.b_start - (nt[1] - na - 1) * kTile};
+            auto valid_of = [&](int x, int j) { return (j == na - 1) ? a_last : (j == nt[x] - 1) ? b_last[x] : kTile; };
+            auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
+            auto wait_full = [&](int idx) {
+                const int g = ring_base + idx;
+                PROF_LAP(5)
+                wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWaitFull);
+                PROF_LAP(2)
+            };
+            auto commit_empty = [&](int idx) { mma_commit_elect(bar_empty + 8 * ((ring_base + idx) % kRing)); };
+            // S_x = Q_x K(j)^T
+            auto issue_qk = [&](int x, int j) {
+                const int n_mma = (valid_of(x, j) + 15) & ~15;
+                const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
+                PROF_LAP(5)
+                mma_ss_batch<D / 16>(tmem_base + x * 128, desc_lo(smem_base + (x ? L::kQ1 : L::kQ0), 16),
+                                     desc_lo(ring_addr(2 * j), 16), idesc);
+                PROF_LAP(6)
+                mma_commit_elect(bar_s_full + 8 * x);
+                if (j == nt[x] - 1) mma_commit_elect(bar_q_free + 8 * x);  // last use of this Q tile
+                PROF_LAP(7)
+            };
+            // O_x += P_x V(j)
+            auto issue_pv = [&](int x, int j) {
+                PROF_LAP(5)
+                wait(bar_po + 8 * x, (cnt[x] + j) & 1, kWaitPO);
+                PROF_LAP(3)
+                // the previous item's output must have left TMEM before O is overwritten
+                if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWaitOFree);
+                PROF_LAP(4)
+                tc_fence_after_sync();
+                const int nvalid = valid_of(x, j);
+                const uint32_t idesc = make_idesc_bf16(kTile, D, true);
+                const uint32_t sv = ring_addr(2 * j + 1);
+                const uint32_t d_tmem = tmem_base + 256 + x * 128, a_tmem = tmem_base + x * 128;
+                PROF_LAP(5)
+                if (nvalid == kTile) {
+                    mma_ts_batch8(d_tmem, a_tmem, desc_lo(sv, L::kPanelBytes), idesc, j > 0);
+                } else {
+                    const int ksteps = (nvalid + 15) >> 4;
+                    for (int ks = 0; ks < ksteps; ++ks)
+                        mma_ts_elect(d_tmem, a_tmem + ks * 8, make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc,
+                                     (j > 0) || (ks > 0));
+                }
+                PROF_LAP(1)
+                // pv: read by the softmax for its rare in-place rescale (one phase per tile);
+                // o_done: the item's accumulator is complete (one phase per item, for the epilogue)
+                mma_commit_elect(bar_pv + 8 * x);
+                if (j == nt[x] - 1) mma_commit_elect(bar_o_done + 8 * x);
+                PROF_LAP(7)
+            };
+            PROF_LAP(5)
+#pragma unroll
+            for (int x = 0; x < 2; ++x)
+                if (nt[x] > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWaitQ);
+            PROF_LAP(4)
             tc_fence_after_sync();
-            if (tid == 0 && i + 1 < nt) issue_kv_loads(i + 1);
-            if (__any_sync(0xffffffffu, alpha != 1.f)) {
+            // order on the tensor pipe: QK0(j) PV1(j-1) QK1(j) PV0(j): while one query tile is in its
+            // softmax the other one's MMAs run
+            for (int j = 0; j <= nt_max; ++j) {
+                if (j < nt_max) {
+                    wait_full(2 * j);
+                    tc_fence_after_sync();
+                    if (j < nt[0]) issue_qk(0, j);
+                }
+                if (j > 0) {
+                    if (j - 1 < nt[1]) {
+                        wait_full(2 * (j - 1) + 1);
+                        issue_pv(1, j - 1);
+                    }
+                    commit_empty(2 * (j - 1) + 1);  // V(j-1) consumed
+                }
+                if (j < nt_max) {
+                    if (j < nt[1]) issue_qk(1, j);
+                    commit_empty(2 * j);  // K(j) consumed
+                    if (j < nt[0]) {
+                        wait_full(2 * j + 1);
+                        issue_pv(0, j);
+                    }
+                }
+            }
+            ring_base += 2 * nt_max;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                cnt[x] += nt[x];
+                if (nt[x] > 0) ++q_uses[x];
+            }
+        }
+        if (lane == 0) { PROF_DUMP(0, 8) }
+      }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------- softmax of slot x
+        reg_alloc<200>();
+        const int x = warp >> 2;
+        const int row = tid & 127;
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + x * 128 + lane_off;
+        const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
+        const uint32_t my_s_full = bar_s_full + 8 * x, my_po = bar_po + 8 * x, my_pv = bar_pv + 8 * x;
+        int cnt = 0;   // tiles of this slot processed so far (phase of s_full / pv)
+        int uses = 0;  // items in which this slot was active so far
+        PROF_DECL(8)
+        for (int k = 0;; ++k) {
+            PROF_LAP(7)
+            const int w = next_item(k);
+            PROF_LAP(0)
+            if (w < 0) break;
+            WorkItem it;
+            decode_item(p, w, it);
+            // this slot's scalars, in registers
+            const int nt = x ? it.s[1].nt : it.s[0].nt;
+            if (nt == 0) continue;
+            const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
+            const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
+            const int na = it.na, a_end = it.a_end, b_start = it.b_start;
+            const int my_limit = limit0 + row / it.row_div;
+            float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
+            float l_run = 0.f;
+            for (int j = 0; j < nt; ++j, ++cnt) {
+                const int j0 = j < na ? j * kTile : b_start + (j - na) * kTile;
+                const int nvalid = min(kTile, (j < na ? a_end : b_end) - j0);
+                const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > limit0);
+                PROF_LAP(7)
+                wait(my_s_full, cnt & 1, kWaitS);
+                PROF_LAP(1)
+                tc_fence_after_sync();
+                // all 128 scores of the row in registers: one round trip to TMEM
+                uint32_t r[kTile];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
+                tmem_wait_ld();
+                PROF_LAP(2)
+                if (need_mask) {
+                    const int max_col = min(nvalid, my_limit - j0 + 1);
+#pragma unroll
+                    for (int i = 0; i < kTile; ++i)
+                        if (i >= max_col) r[i] = 0xff800000u;  // -inf
+                }
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int i = 0; i < kTile; i += 8) {
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+                        mx[a] = fmax3(mx[a], __uint_as_float(r[i + 2 * a]), __uint_as_float(r[i + 2 * a + 1]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                float alpha = 1.f;
+                if ((m_tile - m_ref) * p.scale_log2 > kRescaleThresholdLog2 || m_ref == -INFINITY) {
+                    const float m_new = fmaxf(m_ref, m_tile);
+                    alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
+                    m_ref = m_new;
+                }
+                PROF_LAP(3)
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    // rare: rescale this row of the O accumulator in place, once PV(j-1) has landed.
+                    // (S(j) is complete, so PV(j-2) is too: the wait is at most one phase behind.)
+                    wait(my_pv, (cnt - 1) & 1, kWaitPV);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                }
+                PROF_LAP(4)
+                const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
+                // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot);
+                // scale-and-shift and the row sum run as packed fp32 pairs
+                const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+                const uint64_t shift2 = pack_f32x2(neg_ms, neg_ms);
+                uint64_t sm2[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint64_t t2 = fma_f32x2(pack_f32x2(__uint_as_float(r[c * 32 + 2 * i]),
+                                                                 __uint_as_float(r[c * 32 + 2 * i + 1])), scale2, shift2);
+                        float t0, t1;
+                        unpack_f32x2(t2, t0, t1);
+                        const float p0 = fast_exp2(t0), p1 = fast_exp2(t1);
+                        sm2[i & 3] = add_f32x2(sm2[i & 3], pack_f32x2(p0, p1));
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                float sum;
+                {
+                    float a0, a1, b0, b1;
+                    unpack_f32x2(add_f32x2(sm2[0], sm2[1]), a0, a1);
+                    unpack_f32x2(add_f32x2(sm2[2], sm2[3]), b0, b1);
+                    sum = (a0 + a1) + (b0 + b1);
+                }
+                PROF_LAP(5)
+                tmem_wait_st();
+                PROF_LAP(6)
+                tc_fence_before_sync();
+                mbar_arrive(my_po);
+                l_run = l_run * alpha + sum;
+            }
+            s_final_l[uses & 1][x][row] = l_run;
+            s_final_m[uses & 1][x][row] = m_ref;
+            mbar_arrive(bar_final + 8 * x);
+            ++uses;
+        }
+        if (tid == 0 || tid == 128) { PROF_DUMP(8 + 8 * x, 8) }
+    } else {
+        // ------------------------------------------------------------- epilogue
+        reg_dealloc<64>();
+        const int row = tid & 127;
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_done / o_free)
+        for (int k = 0;; ++k) {
+            const int w = next_item(k);
+            if (w < 0) break;
+            WorkItem it;
+            decode_item(p, w, it);
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                const QSlot& s = it.s[x];
+                if (!s.valid) continue;
+                const bool row_ok = row < s.rows_valid;
+                const int tok = s.q_tok0 + row / it.row_div;
+                const int head = s.q_head0 + row % it.row_div;
+                if (s.nt == 0) {
+                    // question-mode slot with no visible key in this CTA's key range: neutral partial
+                    if (p.mode == 1 && row_ok) {
+                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                        p.part_lse[r] = -INFINITY;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+                        for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    continue;
+                }
+                wait(bar_final + 8 * x, uses[x] & 1, kWaitFinal);
+                const float l = s_final_l[uses[x] & 1][x][row], m = s_final_m[uses[x] & 1][x][row];
+                wait(bar_o_done + 8 * x, uses[x] & 1, kWaitPV);
+                tc_fence_after_sync();
+                const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+                const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
+                const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
-                    uint32_t orow[32];
-                    tmem_ld32(tO + lane_off + c * 32, orow);
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
                     tmem_wait_ld();
+                    if (c == D / 32 - 1) {
+                        // every column of this row is in registers: the accumulator may be reused
+                        tc_fence_before_sync();
+                        mbar_arrive(bar_o_free + 8 * x);
+                    }
+                    if (!row_ok) continue;
+                    if (p.mode == 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
-                    tmem_st32(tO + lane_off + c * 32, orow);
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t wd[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                wd[e] = pack_bf16x2(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
+                                                    __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
+                            dst[v] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                        }
+                    } else {
+                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D + c * 32);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
+                                                 __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                    }
+                }
+                if (row_ok) {
+                    if (p.mode == 0) {
+                        if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
+                    } else {
+                        p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+                    }
                 }
             }
-        }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_st16(tP + lane_off + c * 16, pk + c * 16);
-        tmem_wait_st();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after_sync();
-            if (!mbar_wait(bar_v0 + 8 * s, (i / kStages) & 1, &abort_flag)) give_up(kWaitV);
-            issue_pv(i);
-            if (i + 1 < nt) {
-                if (!mbar_wait(bar_k0 + 8 * ((i + 1) % kStages), ((i + 1) / kStages) & 1, &abort_flag)) give_up(kWaitK);
-                issue_qk(i + 1);
-            }
-        }
-    }
-
-    if (!mbar_wait(bar_o, (nt - 1) & 1, &abort_flag)) give_up(kWaitO);
-    tc_fence_after_sync();
-
-    // epilogue: O / l -> bf16 (prefill) or fp32 partial (question), LSE = m * scale + ln l
-    const bool row_ok = tid < it.rows_valid;
-    const int tok = it.q_tok0 + tid / it.row_div;
-    const int head = it.q_head0 + tid % it.row_div;
-    const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-    const float lse_val = (l_run > 0.f) ? m_run * p.scale + logf(l_run) : -INFINITY;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t orow[32];
-        tmem_ld32(tO + lane_off + c * 32, orow);
-        tmem_wait_ld();
-        if (row_ok) {
-            if (p.mode == 0) {
-                uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        w[e] = pack_bf16x2(__uint_as_float(orow[v * 8 + 2 * e]) * inv_l,
-                                           __uint_as_float(orow[v * 8 + 2 * e + 1]) * inv_l);
-                    dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-            } else {
-                const size_t row = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-                float4* dst = reinterpret_cast<float4*>(p.part_o + row * D + c * 32);
-#pragma unroll
-                for (int v = 0; v < 8; ++v)
-                    dst[v] = make_float4(__uint_as_float(orow[v * 4]) * inv_l, __uint_as_float(orow[v * 4 + 1]) * inv_l,
-                                         __uint_as_float(orow[v * 4 + 2]) * inv_l, __uint_as_float(orow[v * 4 + 3]) * inv_l);
-            }
-        }
-    }
-    if (row_ok) {
-        if (p.mode == 0) {
-            if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
-        } else {
-            p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+            for (int x = 0; x < 2; ++x)
+                if (it.s[x].nt > 0) ++uses[x];
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
-}
-
-// Merge of key-range partials: lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s.
-// One thread per (row, 4 output columns).
-__global__ void merge_kernel(const __grid_constant__ MergeParams p) {
-    const int vec_per_row = p.d / 4;
-    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int64_t rows = static_cast<int64_t>(p.Q) * p.Hq;
-    if (idx >= rows * vec_per_row) return;
-    const int64_t row = idx / vec_per_row;  // = tok * Hq + head
-    const int v = static_cast<int>(idx % vec_per_row);
-    float m = -INFINITY;
-    for (int s = 0; s < p.n_splits; ++s) m = fmaxf(m, p.part_lse[s * rows + row]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float l = 0.f;
-    if (m != -INFINITY) {
-        for (int s = 0; s < p.n_splits; ++s) {
-            const float ls = p.part_lse[s * rows + row];
-            if (ls == -INFINITY) continue;
-            const float w = __expf(ls - m);
-            l += w;
-            const float4 o = reinterpret_cast<const float4*>(p.part_o + (s * rows + row) * p.d)[v];
-            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
-        }
-    }
-    const float inv = (l > 0.f) ? 1.f / l : 0.f;
-    uint2 out;
-    out.x = pack_bf16x2(acc.x * inv, acc.y * inv);
-    out.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-    reinterpret_cast<uint2*>(p.o + row * p.d)[v] = out;
-    if (p.lse && v == 0) {
-        const int tok = static_cast<int>(row / p.Hq), head = static_cast<int>(row % p.Hq);
-        p.lse[static_cast<int64_t>(head) * p.Q + tok] = (l > 0.f) ? m + logf(l) : -INFINITY;
+    if (warp == 12) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
 cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
-                        const CUtensorMap& tv, cudaStream_t stream) {
+                           const CUtensorMap& tv, cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
     const size_t smem = attn_smem_bytes(head_dim);
-    cudaError_t e;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int grid = p.n_items < sms ? p.n_items : sms;  // persistent: one CTA per SM
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<128><<<p.n_items, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_kernel<128><<<grid, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
     } else {
         e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<64><<<p.n_items, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_kernel<64><<<grid, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
     }
-    return cudaGetLastError();
-}
-
-cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream) {
-    const int64_t n = static_cast<int64_t>(p.Q) * p.Hq * (p.d / 4);
-    if (n <= 0) return cudaSuccess;
-    merge_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -30,10 +30,10 @@ struct AttnParams {
     int32_t Hq, Hkv, G;
     int32_t tiles_sink;     // ceil(S / 128)
     int32_t tiles_block;    // ceil(B / 128)
-    int32_t items_block;    // N * tiles_block * Hq
-    int32_t n_items;        // grid size
-    int32_t pairs_block;    // paired kernel: ceil(G * tiles_block / 2) query-tile pairs per (block, kv head)
-    int32_t pairs_sink;     // paired kernel: ceil(G * tiles_sink / 2)
+    int32_t pairs_block;    // ceil(G * tiles_block / 2) query-tile pairs per (block, kv head)
+    int32_t pairs_sink;     // ceil(G * tiles_sink / 2) query-tile pairs per kv head
+    int32_t items_block;    // N * Hkv * pairs_block work items over the context blocks
+    int32_t n_items;        // all work items of the launch
     int32_t q_box_rows;     // rows the Q TMA box brings in (128 prefill, G * tok_per_tile question)
     int32_t tok_per_tile;   // mode 1: question tokens per query tile = 128 / G
     int32_t q_tiles;        // mode 1: ceil(Q / tok_per_tile)
@@ -80,9 +80,6 @@ cudaError_t launch_copy_segments(const CopySegments& s, cudaStream_t stream);
 cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
                         const CUtensorMap& tv, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
-cudaError_t launch_attn_ws(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
-                           const CUtensorMap& tv, cudaStream_t stream);
 size_t attn_smem_bytes(int head_dim);
-size_t attn_ws_smem_bytes(int head_dim);
 
 }  // namespace pevlm

@@ -120,6 +120,33 @@ int pevlm_query_attn(const pevlm_shape_t* shape, const void* q_question, const v
                      const void* v_cache, void* o, float* lse, void* workspace,
                      size_t workspace_bytes, void* stream);
 
+/*
+ * Question attention without a caller workspace.  (The paper has no counterpart to this entry
+ * point; it exists for deployment.)
+ *
+ * For callers that cannot allocate device memory where they need this step -- code inside a
+ * memory-planned or real-time region that must not call cudaMalloc or any allocating library
+ * routine, or a plug-in that is handed inputs and outputs but owns no memory pool.  Same
+ * arguments, results and errors as pevlm_query_attn, minus the workspace: the split-KV partials
+ * go to a fixed array of PEVLM_NOALLOC_SCRATCH_BYTES that is part of the library image, so
+ * every GPU that loads the library holds that much device memory until the process exits.
+ *   - Shapes whose pevlm_workspace_bytes(shape, PEVLM_WS_QUERY) exceeds that size are rejected
+ *     with PEVLM_EWORKSPACE before any launch (text via pevlm_last_cuda_error).
+ *   - The call itself performs no cudaMalloc / cudaFree and uses no allocating routine.
+ *   - The first call on each device resolves the array's device address
+ *     (cudaGetSymbolAddress, with that device current); make that first call outside any
+ *     stream capture.
+ *   - All calls on one device share the one array, which keeps the previous call's contents:
+ *     each call clears the status header it needs on the stream and overwrites the partials it
+ *     reads.  Two calls whose kernels overlap on the GPU (different streams, no ordering
+ *     between them) race on the array; order them.
+ *   - A device-side timeout is left in the array's header; it cannot be read back through
+ *     pevlm_read_status, which takes a caller workspace.
+ */
+#define PEVLM_NOALLOC_SCRATCH_BYTES (32u << 20)
+int pevlm_query_attn_noalloc(const pevlm_shape_t* shape, const void* q_question, const void* k_cache,
+                             const void* v_cache, void* o, float* lse, void* stream);
+
 /* Bytes of workspace the given call needs for this shape (0 if the shape is invalid). */
 size_t pevlm_workspace_bytes(const pevlm_shape_t* shape, int which /* pevlm_workspace_kind_t */);
 

@@ -19,7 +19,10 @@ PEVLM_EINVAL, PEVLM_EALIGN, PEVLM_EUNSUPPORTED, PEVLM_EWORKSPACE, PEVLM_ECUDA, P
 MASK_PEVLM, MASK_FULL_CAUSAL = 0, 1
 WS_PREFILL, WS_QUERY = 0, 1
 
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
 EXPORTS = ["pevlm_rope_qk", "pevlm_parallel_prefill_attn", "pevlm_assemble_kv", "pevlm_query_attn",
+           "pevlm_query_attn_noalloc",
            "pevlm_workspace_bytes", "pevlm_read_status", "pevlm_tile_stats", "pevlm_strerror",
            "pevlm_last_cuda_error"]
 
@@ -67,6 +70,8 @@ def lib():
         l.pevlm_parallel_prefill_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         l.pevlm_assemble_kv.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp]
         l.pevlm_query_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        l.pevlm_query_attn_noalloc.argtypes = [sp, vp, vp, vp, vp, vp, vp]
+        l.pevlm_query_attn_noalloc.restype = C.c_int
         l.pevlm_workspace_bytes.argtypes = [sp, C.c_int]
         l.pevlm_workspace_bytes.restype = C.c_size_t
         l.pevlm_read_status.argtypes = [vp, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -119,6 +124,13 @@ def pevlm_query_attn(shape: Shape, q_question, k_cache, v_cache, o, lse, workspa
     _check(lib().pevlm_query_attn(C.byref(shape), _ptr(q_question), _ptr(k_cache), _ptr(v_cache), _ptr(o),
                                   _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                   _stream()), "pevlm_query_attn")
+
+
+def pevlm_query_attn_noalloc(shape: Shape, q_question, k_cache, v_cache, o, lse):
+    """Question attention for callers that cannot allocate device memory: no workspace argument,
+    the partials go to the library's built-in scratch array (see include/pevlm.h for its limits)."""
+    _check(lib().pevlm_query_attn_noalloc(C.byref(shape), _ptr(q_question), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                          _ptr(lse), _stream()), "pevlm_query_attn_noalloc")
 
 
 def pevlm_read_status(workspace):

@@ -14,7 +14,7 @@ import sys
 _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
 LIB = os.path.join(_DIR, "libpevlm.so")
-SOURCES = ["api.cu", "rope_kernel.cu", "assemble_kernel.cu", "attn_kernel.cu", "merge_kernel.cu"]
+SOURCES = ["api.cu", "rope_kernel.cu", "assemble_kernel.cu", "attn_kernel.cu", "merge_kernel.cu", "query_noalloc.cu"]
 HEADERS = ["internal.h", "ptx.cuh", os.path.join("..", "..", "include", "pevlm.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]

@@ -11,9 +11,14 @@ namespace pevlm {
 
 static thread_local char g_cuda_error[256] = "";
 
-static int cuda_fail(cudaError_t e, const char* what) {
+int cuda_fail(cudaError_t e, const char* what) {
     snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
     return PEVLM_ECUDA;
+}
+
+int fail_with_text(int code, const char* text) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s", text);
+    return code;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

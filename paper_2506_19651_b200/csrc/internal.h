@@ -81,5 +81,9 @@ cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq
                         const CUtensorMap& tv, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 size_t attn_smem_bytes(int head_dim);
+// error reporting shared by the host-side translation units: both record a text that
+// pevlm_last_cuda_error returns on the calling thread
+int cuda_fail(cudaError_t e, const char* what);      // returns PEVLM_ECUDA
+int fail_with_text(int code, const char* text);      // returns code
 
 }  // namespace pevlm

@@ -153,7 +153,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     constexpr int NP = L::kPanels;
     extern __shared__ uint8_t smem_raw[];
     // barrier map (uint64 each): [0,2) item_full [2,4) item_free [4,6) q_full [6,8) q_free
-    // [8,12) ring full [12,16) ring empty, then per slot x: [16,18) s_full [18,20) po [20,22) pv
+    // [8,12) ring full [12,16) ring empty, then per slot x: [16,18) s_full [18,20) po
     // [22,24) final [24,26) o_free [26,28) o_done
     __shared__ uint64_t bars[28];
     __shared__ uint32_t tmem_base_slot;
@@ -169,7 +169,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     const uint32_t bar0 = smem_u32(&bars[0]);
     const uint32_t bar_item_full = bar0, bar_item_free = bar0 + 16, bar_q_full = bar0 + 32, bar_q_free = bar0 + 48;
     const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
-    const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144, bar_pv = bar0 + 160;
+    const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144;
     const uint32_t bar_final = bar0 + 176, bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
     constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA warp + two softmax warpgroups + epilogue warpgroup
 
@@ -182,7 +182,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             mbar_init(bar_q_free + 8 * i, 1);
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_po + 8 * i, kTile);
-            mbar_init(bar_pv + 8 * i, 1);
             mbar_init(bar_final + 8 * i, kTile);
             mbar_init(bar_o_free + 8 * i, kTile);
             mbar_init(bar_o_done + 8 * i, 1);
@@ -268,7 +267,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         // All 32 lanes run this loop with warp-uniform values (descriptors and addresses stay in
         // uniform registers); the MMA and commit instructions themselves go out from one elected lane.
         int ring_base = 0;        // ring position of this item's K(0)
-        int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po / pv)
+        int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po)
         int q_uses[2] = {0, 0};   // items in which the slot was active so far
         PROF_DECL(8)
         for (int k = 0;; ++k) {
@@ -334,9 +333,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                                      (j > 0) || (ks > 0));
                 }
                 PROF_LAP(1)
-                // pv: read by the softmax for its rare in-place rescale (one phase per tile);
                 // o_done: the item's accumulator is complete (one phase per item, for the epilogue)
-                mma_commit_elect(bar_pv + 8 * x);
                 if (j == nt[x] - 1) mma_commit_elect(bar_o_done + 8 * x);
                 PROF_LAP(7)
             };
@@ -387,9 +384,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + x * 128 + lane_off;
         const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
-        const uint32_t my_s_full = bar_s_full + 8 * x, my_po = bar_po + 8 * x, my_pv = bar_pv + 8 * x;
-        int cnt = 0;   // tiles of this slot processed so far (phase of s_full / pv)
-        int uses = 0;  // items in which this slot was active so far
+        const uint32_t my_s_full = bar_s_full + 8 * x, my_po = bar_po + 8 * x;
+        int cnt = 0;        // tiles of this slot processed so far (phase of s_full)
+        int uses = 0;       // items in which this slot was active so far
+        int ring_base = 0;  // ring position of this item's K(0)
         PROF_DECL(8)
         for (int k = 0;; ++k) {
             PROF_LAP(7)
@@ -400,6 +398,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             decode_item(p, w, it);
             // this slot's scalars, in registers
             const int nt = x ? it.s[1].nt : it.s[0].nt;
+            const int item_ring_base = ring_base;
+            ring_base += 2 * max(it.s[0].nt, it.s[1].nt);
             if (nt == 0) continue;
             const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
             const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
@@ -443,9 +443,11 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 }
                 PROF_LAP(3)
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                    // rare: rescale this row of the O accumulator in place, once PV(j-1) has landed.
-                    // (S(j) is complete, so PV(j-2) is too: the wait is at most one phase behind.)
-                    wait(my_pv, (cnt - 1) & 1, kWaitPV);
+                    // rare: rescale this row of the O accumulator in place, once PV(j-1) has landed: the
+                    // ring slot of V(j-1) is released by a commit issued after both slots' PV(j-1).
+                    // (S(j) is complete, so that slot's previous release, two tiles back, is too.)
+                    const int gv = item_ring_base + 2 * (j - 1) + 1;
+                    wait(bar_empty + 8 * (gv % kRing), (gv / kRing) & 1, kWaitPV);
                     tc_fence_after_sync();
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
@@ -493,6 +495,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 mbar_arrive(my_po);
                 l_run = l_run * alpha + sum;
             }
+            // A one-tile item never waits for the previous item's epilogue on its way here: hold the
+            // `final` arrival until that epilogue has consumed the previous one (it signals o_free after
+            // reading it), so the barrier never runs two phases ahead of its waiter.
+            if (uses > 0) wait(bar_o_free + 8 * x, (uses - 1) & 1, kWaitOFree);
             s_final_l[uses & 1][x][row] = l_run;
             s_final_m[uses & 1][x][row] = m_ref;
             mbar_arrive(bar_final + 8 * x);

@@ -196,6 +196,7 @@ def run_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_2506_19651_b200 import binding as pb
+    from paper_2506_19651_b200 import replicas
     from paper_2506_19651_b200.layer import KERNELS_PER_PASS, LayerBuffers, layer_forward
 
     rank = int(os.environ.get("RANK", "0"))
@@ -224,11 +225,7 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, device="cuda")
 
     names = ["rope_video", "assemble_video", "prefill_attn", "rope_question", "assemble_question", "query_attn"]
 
@@ -328,7 +325,7 @@ def run_ours(args, w):
     achieved = pre.flops / (t_pre * 1e-3) / 1e12
     kv_bytes = 2.0 * w.L * w.Hkv * w.d * 2
     line = {
-        "metric": METRIC, "value": world * flops_layer / (ms_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": replicas.whole_job_rate(flops_layer, world, ms_step) / 1e12, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": dict(workload_config(w), parallelism="replicas" if world > 1 else "single GPU"),
@@ -344,7 +341,7 @@ def run_ours(args, w):
         "roofline": {"kernel": "attn_kernel (pevlm_parallel_prefill_attn)", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "peak_source": peaks["source"] + " (burst bf16 GEMM)", "traffic": None},
-        "e2e": {"value": world * flops_layer / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": replicas.whole_job_rate(flops_layer, world, e2e_ms) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": KERNELS_PER_PASS * args.steps,
         "clocks": clocks,

@@ -146,3 +146,69 @@ def test_full_size_sampled_rows(name, n_random):
     np.testing.assert_array_equal(res["v_cache"], v)
     for key, e in errs.items():
         assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)
+
+
+# ---------------------------------------------------------------- batch > 1 (independent sequences)
+
+def test_batch_of_two_sequences():
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(96, 160, 2, 24, 4, 2, 128, outliers=True)
+    nv = w.n_video
+    seqs = [inputs.make_qkv(w.with_(seed=w.seed + i)) for i in range(2)]
+    s = gpu_shape(w)
+    s.batch = 2
+    cat = lambda idx, sl: to_dev(np.concatenate([seqs[b][idx][sl] for b in range(2)], axis=0))
+    q_v, k_v, v_v = cat(0, slice(0, nv)), cat(1, slice(0, nv)), cat(2, slice(0, nv))
+    q_q, k_q, v_q = cat(0, slice(nv, None)), cat(1, slice(nv, None)), cat(2, slice(nv, None))
+    pb.pevlm_rope_qk(s, q_v, k_v, q_v, k_v, 0, nv)
+    pb.pevlm_rope_qk(s, q_q, k_q, q_q, k_q, nv, w.Q)
+    kc = torch.empty((2 * w.L, w.Hkv, w.d), dtype=torch.bfloat16, device="cuda")
+    vc = torch.empty_like(kc)
+    pb.pevlm_assemble_kv(s, k_v, v_v, k_q, v_q, kc, vc)
+    o_v = torch.empty_like(q_v)
+    lse_v = torch.empty((2, w.Hq, nv), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device="cuda")
+    pb.pevlm_parallel_prefill_attn(s, q_v, k_v, v_v, o_v, lse_v, ws)
+    o_q = torch.empty_like(q_q)
+    lse_q = torch.empty((2, w.Hq, w.Q), dtype=torch.float32, device="cuda")
+    wq = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device="cuda")
+    pb.pevlm_query_attn(s, q_q, kc, vc, o_q, lse_q, wq)
+    torch.cuda.synchronize()
+    assert pb.pevlm_read_status(ws)[0] == 0 and pb.pevlm_read_status(wq)[0] == 0
+    for b in range(2):
+        q, k, v = seqs[b]
+        qr, kr = oracle.rope(q, w.theta), oracle.rope(k, w.theta)
+        np.testing.assert_array_equal(to_bits(kc[b * w.L:(b + 1) * w.L]), kr)
+        np.testing.assert_array_equal(to_bits(vc[b * w.L:(b + 1) * w.L]), v)
+        sh = oracle.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d)
+        o_ref, lse_ref = oracle.attn_rows(sh, qr, kr, v, np.arange(w.L))
+        got_o = np.concatenate([bits_to_f64(to_bits(o_v[b * nv:(b + 1) * nv])), bits_to_f64(to_bits(o_q[b * w.Q:(b + 1) * w.Q]))])
+        got_l = np.concatenate([lse_v[b].double().cpu().numpy().T, lse_q[b].double().cpu().numpy().T])
+        assert np.abs(got_o - o_ref).max() <= O_TOL
+        assert np.abs(got_l - lse_ref).max() <= LSE_TOL
+
+
+# ---------------------------------------------------------------- the other full-size configurations
+
+@pytest.mark.parametrize("name,n_random", [("c4_sweep_F1", 200), ("c4_sweep_F32", 60), ("c5_stack", 60)])
+def test_sweep_and_stack_sampled_rows(name, n_random):
+    w = inputs.WORKLOADS[name]
+    q, k, v = inputs.make_qkv(w, layer=13 if w.layers > 1 else 0)
+    res = run_gpu_layer(w, q, k, v)
+    rows = inputs.sample_rows(w, n_random)
+    errs, qr, kr = check_against_oracle(w, q, k, v, res, rows)
+    assert int((res["k_cache"] != kr).sum()) <= 2
+    for key, e in errs.items():
+        assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)
+
+
+def test_full_causal_mode_full_size_sampled_rows():
+    # the speed-up baseline: plain causal attention over the 12,544 video tokens of the Qwen-shaped layer
+    w = inputs.WORKLOADS["c2_qwen"]
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v, full_causal=True)
+    rows = inputs.sample_rows(w, 100)
+    errs, _, _ = check_against_oracle(w, q, k, v, res, rows[rows < w.n_video], full_causal=True)
+    for key, e in errs.items():
+        assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)

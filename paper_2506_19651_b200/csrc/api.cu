@@ -109,8 +109,12 @@ static QueryPlan plan_query(const pevlm_shape_t* s) {
     q.tok_per_tile = kTile / G;
     q.q_tiles = (s->query_len + q.tok_per_tile - 1) / q.tok_per_tile;
     q.total_kv_tiles = static_cast<int>((L + kTile - 1) / kTile);
-    const int groups = s->num_kv_heads * (q.q_tiles > 0 ? q.q_tiles : 1);
-    int want = (2 * 148 + groups - 1) / groups;  // about two CTAs per SM
+    // Work items are (kv head, pair of query tiles, key split).  The kernel is persistent with one
+    // CTA per SM, so the split count is chosen to give one full wave of the 148 SMs of a B200:
+    // as many splits as fit, never more than there are key tiles.
+    const int pairs = (q.q_tiles + 1) / 2;
+    const int groups = s->num_kv_heads * (pairs > 0 ? pairs : 1);
+    int want = kNumSms / groups;
     if (want < 1) want = 1;
     if (want > q.total_kv_tiles) want = q.total_kv_tiles;
     q.tiles_per_split = (q.total_kv_tiles + want - 1) / want;

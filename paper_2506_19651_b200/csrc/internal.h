@@ -11,6 +11,7 @@ namespace pevlm {
 
 constexpr int kTile = 128;        // query-tile rows (MMA M) and key-tile columns (MMA N max)
 constexpr int kStatusBytes = 256; // first bytes of every workspace: status word + detail + counters
+constexpr int kNumSms = 148;      // B200; used only to size the key splits of the question attention
 
 // Workspace header (device memory, first kStatusBytes of the workspace).
 struct WorkspaceHeader {

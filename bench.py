@@ -358,6 +358,107 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def device_inputs(w, layer=0):
+    """Un-roped bf16 Q, K, V generated on the device (seeded): same distribution as inputs.make_qkv
+    (N(0,1), first four sink K rows x8 when the workload has outliers), used where 28 layers of host
+    generation would take minutes.  Parity is never checked on these; the tests use inputs.make_qkv."""
+    import torch
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed + layer)
+    mk = lambda h: torch.randn((w.L, h, w.d), generator=g, device="cuda", dtype=torch.float32)
+    q, k, v = mk(w.Hq), mk(w.Hkv), mk(w.Hkv)
+    if w.outliers:
+        k[:min(4, w.S)] *= 8.0
+    return q.bfloat16(), k.bfloat16(), v.bfloat16()
+
+
+def time_layer(w, steps, warmup, q, k, v, buf=None):
+    """Per-kernel milliseconds of `steps` passes over one layer (CUDA events on the current stream)."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    from paper_2506_19651_b200.layer import LayerBuffers, layer_forward
+    shape = pb.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d, theta=w.theta)
+    buf = buf or LayerBuffers(shape)
+    for _ in range(warmup):
+        layer_forward(buf, q, k, v)
+    torch.cuda.synchronize()
+    marks = []
+
+    def mark(name):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        marks.append((name, ev))
+
+    for _ in range(steps):
+        layer_forward(buf, q, k, v, mark=mark)
+    torch.cuda.synchronize()
+    per = {}
+    for (n0, e0), (n1, e1) in zip(marks[:-1], marks[1:]):
+        if n1 != "start":
+            per[n1] = per.get(n1, 0.0) + e0.elapsed_time(e1) / steps
+    for ws in (buf.ws_prefill, buf.ws_query):
+        st, det = pb.pevlm_read_status(ws)
+        if st != 0:
+            raise RuntimeError(f"device wait expired: status {st} detail {det}")
+    return shape, per
+
+
+def run_sweep(args):
+    """Block-size sweep (128 frames x 256 tokens, sink = one block of F frames): one JSON line per F."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    for F in (1, 2, 4, 8, 16, 32):
+        w = inputs.sweep_workload(F)
+        q, k, v = device_inputs(w)
+        shape, per = time_layer(w, args.steps, args.warmup, q, k, v)
+        pre = pb.pevlm_tile_stats(shape, pb.WS_PREFILL)
+        t = per["prefill_attn"]
+        useful = 4.0 * w.d * w.Hq * (visible_pairs(w) - (w.Q * w.n_video + w.Q * (w.Q + 1) // 2))
+        fshape = pb.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d, theta=w.theta, mask_mode=pb.MASK_FULL_CAUSAL)
+        print(json.dumps({"kind": "sweep", "workload": w.name, "frames_per_block": F, "block_len": w.B, "num_blocks": w.N,
+                          "ms_per_layer": sum(per.values()), "kernels_ms": per, "prefill_ms": t,
+                          "active_tile_tflops": pre.flops / (t * 1e-3) / 1e12, "useful_tflops": useful / (t * 1e-3) / 1e12,
+                          "frac_of_bf16_peak": pre.flops / (t * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                          "full_causal_active_gflop": pb.pevlm_tile_stats(fshape, pb.WS_PREFILL).flops / 1e9,
+                          "data": "synthetic (device-generated)"}))
+
+
+def run_stack(args):
+    """Attention of a whole prefill stack: every layer has its own seeded Q/K/V and its own KV cache."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    from paper_2506_19651_b200.layer import LayerBuffers, layer_forward
+    torch.cuda.set_device(0)
+    w = inputs.WORKLOADS["c5_stack"]
+    layers = args.layers or w.layers
+    shape = pb.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d, theta=w.theta)
+    bufs = [LayerBuffers(shape) for _ in range(layers)]          # one KV cache per layer stays resident
+    # two input sets alternate between layers (28 distinct sets would be 19 GB of inputs on top of the caches)
+    ins = [device_inputs(w, layer=i) for i in range(2)]
+    run = lambda: [layer_forward(bufs[i], *ins[i % 2]) for i in range(layers)]
+    for _ in range(max(1, args.warmup)):
+        run()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        run()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    _, per = time_layer(w, args.steps, 1, *ins[0], buf=bufs[0])
+    cache_bytes = 2 * w.L * w.Hkv * w.d * 2
+    asm_ms = per["assemble_video"] + per["assemble_question"]
+    print(json.dumps({"kind": "stack", "workload": w.name, "layers": layers, "tokens": w.L, "attention_ms_total": ms,
+                      "ms_per_layer": ms / layers, "kernels_ms_layer0": per, "kv_cache_bytes_per_layer": cache_bytes,
+                      "kv_cache_bytes_total": cache_bytes * layers,
+                      "assemble_gbs_v_only": 2.0 * w.L * w.Hkv * w.d * 2 / (asm_ms * 1e-3) / 1e9,
+                      "note": "K is roped straight into its cache slot by pevlm_rope_qk; the assembly call copies V",
+                      "data": "synthetic (device-generated, two input sets alternating over the layers)"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -367,9 +468,16 @@ def main():
     ap.add_argument("--workload", default="c3_long", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--skip-cpu", action="store_true", help="omit the cpu_baseline leg")
     ap.add_argument("--skip-full-causal", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="block-size sweep: one JSON line per block size")
+    ap.add_argument("--stack", action="store_true", help="28-layer attention stack: one JSON line")
+    ap.add_argument("--layers", type=int, default=0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     w = inputs.WORKLOADS[args.workload]
+    if args.sweep:
+        return run_sweep(args)
+    if args.stack:
+        return run_stack(args)
     if args.impl == "reference":
         run_reference(args, w)
     else:

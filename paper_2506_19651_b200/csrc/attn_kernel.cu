@@ -269,15 +269,15 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         int ring_base = 0;        // ring position of this item's K(0)
         int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po)
         int q_uses[2] = {0, 0};   // items in which the slot was active so far
-        PROF_DECL(8)
+#ifdef PEVLM_PROFILE
+        unsigned prof_po = 0, prof_full = 0, prof_t0 = static_cast<unsigned>(clock64()), prof_a = 0;
+#endif
         for (int k = 0;; ++k) {
-            PROF_LAP(5)
             // every lane reads the item, one lane releases the queue slot
             wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
             const int w = s_item[k & 1];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_item_free + 8 * (k & 1));
-            PROF_LAP(0)
             if (w < 0) break;
             WorkItem it;
             decode_item(p, w, it);
@@ -293,37 +293,40 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
             auto wait_full = [&](int idx) {
                 const int g = ring_base + idx;
-                PROF_LAP(5)
+#ifdef PEVLM_PROFILE
+                prof_a = static_cast<unsigned>(clock64());
+#endif
                 wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWaitFull);
-                PROF_LAP(2)
+#ifdef PEVLM_PROFILE
+                prof_full += static_cast<unsigned>(clock64()) - prof_a;
+#endif
             };
             auto commit_empty = [&](int idx) { mma_commit_elect(bar_empty + 8 * ((ring_base + idx) % kRing)); };
             // S_x = Q_x K(j)^T
             auto issue_qk = [&](int x, int j) {
                 const int n_mma = (valid_of(x, j) + 15) & ~15;
                 const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
-                PROF_LAP(5)
                 mma_ss_batch<D / 16>(tmem_base + x * 128, desc_lo(smem_base + (x ? L::kQ1 : L::kQ0), 16),
                                      desc_lo(ring_addr(2 * j), 16), idesc);
-                PROF_LAP(6)
                 mma_commit_elect(bar_s_full + 8 * x);
                 if (j == nt[x] - 1) mma_commit_elect(bar_q_free + 8 * x);  // last use of this Q tile
-                PROF_LAP(7)
             };
             // O_x += P_x V(j)
             auto issue_pv = [&](int x, int j) {
-                PROF_LAP(5)
+#ifdef PEVLM_PROFILE
+                prof_a = static_cast<unsigned>(clock64());
+#endif
                 wait(bar_po + 8 * x, (cnt[x] + j) & 1, kWaitPO);
-                PROF_LAP(3)
+#ifdef PEVLM_PROFILE
+                prof_po += static_cast<unsigned>(clock64()) - prof_a;
+#endif
                 // the previous item's output must have left TMEM before O is overwritten
                 if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWaitOFree);
-                PROF_LAP(4)
                 tc_fence_after_sync();
                 const int nvalid = valid_of(x, j);
                 const uint32_t idesc = make_idesc_bf16(kTile, D, true);
                 const uint32_t sv = ring_addr(2 * j + 1);
                 const uint32_t d_tmem = tmem_base + 256 + x * 128, a_tmem = tmem_base + x * 128;
-                PROF_LAP(5)
                 if (nvalid == kTile) {
                     mma_ts_batch8(d_tmem, a_tmem, desc_lo(sv, L::kPanelBytes), idesc, j > 0);
                 } else {
@@ -332,16 +335,12 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                         mma_ts_elect(d_tmem, a_tmem + ks * 8, make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc,
                                      (j > 0) || (ks > 0));
                 }
-                PROF_LAP(1)
                 // o_done: the item's accumulator is complete (one phase per item, for the epilogue)
                 if (j == nt[x] - 1) mma_commit_elect(bar_o_done + 8 * x);
-                PROF_LAP(7)
             };
-            PROF_LAP(5)
 #pragma unroll
             for (int x = 0; x < 2; ++x)
                 if (nt[x] > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWaitQ);
-            PROF_LAP(4)
             tc_fence_after_sync();
             // order on the tensor pipe: QK0(j) PV1(j-1) QK1(j) PV0(j): while one query tile is in its
             // softmax the other one's MMAs run
@@ -374,7 +373,13 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 if (nt[x] > 0) ++q_uses[x];
             }
         }
-        if (lane == 0) { PROF_DUMP(0, 8) }
+#ifdef PEVLM_PROFILE
+        if (lane == 0 && blockIdx.x == 0) {
+            p.hdr->pad[0] = static_cast<int32_t>((static_cast<unsigned>(clock64()) - prof_t0) >> 4);
+            p.hdr->pad[1] = static_cast<int32_t>(prof_po >> 4);
+            p.hdr->pad[2] = static_cast<int32_t>(prof_full >> 4);
+        }
+#endif
       }
     } else if (warp < 8) {
         // ------------------------------------------------------------- softmax of slot x
@@ -388,11 +393,11 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         int cnt = 0;        // tiles of this slot processed so far (phase of s_full)
         int uses = 0;       // items in which this slot was active so far
         int ring_base = 0;  // ring position of this item's K(0)
-        PROF_DECL(8)
+#ifdef PEVLM_PROFILE
+        unsigned prof_busy = 0, prof_wait = 0, prof_t1 = 0, prof_t2 = static_cast<unsigned>(clock64()), prof_tiles = 0;
+#endif
         for (int k = 0;; ++k) {
-            PROF_LAP(7)
             const int w = next_item(k);
-            PROF_LAP(0)
             if (w < 0) break;
             WorkItem it;
             decode_item(p, w, it);
@@ -411,16 +416,17 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 const int j0 = j < na ? j * kTile : b_start + (j - na) * kTile;
                 const int nvalid = min(kTile, (j < na ? a_end : b_end) - j0);
                 const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > limit0);
-                PROF_LAP(7)
                 wait(my_s_full, cnt & 1, kWaitS);
-                PROF_LAP(1)
+#ifdef PEVLM_PROFILE
+                prof_t1 = static_cast<unsigned>(clock64());
+                prof_wait += prof_t1 - prof_t2;
+#endif
                 tc_fence_after_sync();
                 // all 128 scores of the row in registers: one round trip to TMEM
                 uint32_t r[kTile];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
                 tmem_wait_ld();
-                PROF_LAP(2)
                 if (need_mask) {
                     const int max_col = min(nvalid, my_limit - j0 + 1);
 #pragma unroll
@@ -441,7 +447,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m_ref - m_new) * p.scale_log2);
                     m_ref = m_new;
                 }
-                PROF_LAP(3)
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     // rare: rescale this row of the O accumulator in place, once PV(j-1) has landed: the
                     // ring slot of V(j-1) is released by a commit issued after both slots' PV(j-1).
@@ -459,7 +464,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                         tmem_st32(tO + c * 32, o);
                     }
                 }
-                PROF_LAP(4)
                 const float neg_ms = (m_ref == -INFINITY) ? 0.f : -m_ref * p.scale_log2;
                 // probabilities, written over the scores as bf16 pairs (columns [0, 64) of the slot);
                 // scale-and-shift and the row sum run as packed fp32 pairs
@@ -488,11 +492,14 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     unpack_f32x2(add_f32x2(sm2[2], sm2[3]), b0, b1);
                     sum = (a0 + a1) + (b0 + b1);
                 }
-                PROF_LAP(5)
                 tmem_wait_st();
-                PROF_LAP(6)
                 tc_fence_before_sync();
                 mbar_arrive(my_po);
+#ifdef PEVLM_PROFILE
+                prof_t2 = static_cast<unsigned>(clock64());
+                prof_busy += prof_t2 - prof_t1;
+                ++prof_tiles;
+#endif
                 l_run = l_run * alpha + sum;
             }
             // A one-tile item never waits for the previous item's epilogue on its way here: hold the
@@ -504,7 +511,13 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             mbar_arrive(bar_final + 8 * x);
             ++uses;
         }
-        if (tid == 0 || tid == 128) { PROF_DUMP(8 + 8 * x, 8) }
+#ifdef PEVLM_PROFILE
+        if ((tid == 0 || tid == 128) && blockIdx.x == 0) {
+            p.hdr->pad[8 + 8 * x] = static_cast<int32_t>(prof_busy >> 4);
+            p.hdr->pad[9 + 8 * x] = static_cast<int32_t>(prof_wait >> 4);
+            p.hdr->pad[10 + 8 * x] = static_cast<int32_t>(prof_tiles);
+        }
+#endif
     } else {
         // ------------------------------------------------------------- epilogue
         reg_dealloc<64>();

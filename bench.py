@@ -28,6 +28,10 @@ sys.path.insert(0, ROOT)
 
 from paper_2506_19651_b200 import inputs  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one pevlm_parallel_prefill_attn launch, from the
+# one-pass ncu capture summarised in profiles/dram_traffic_c3_long.md (and the c2_qwen full capture)
+NCU_PREFILL_TRAFFIC_BYTES = {"c3_long": 784.8e6, "c2_qwen": 167.0e6}
+
 METRIC = "active_tile_tflops_per_layer"
 UNIT = "TFLOP/s"
 
@@ -340,7 +344,10 @@ def run_ours(args, w):
         "rope": {"ms": per_kernel["rope_video"], "gbs": 2.0 * w.n_video * (w.Hq + w.Hkv) * w.d * 2 / (per_kernel["rope_video"] * 1e-3) / 1e9},
         "roofline": {"kernel": "attn_kernel (pevlm_parallel_prefill_attn)", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                     "peak_source": peaks["source"] + " (burst bf16 GEMM)", "traffic": None},
+                     "peak_source": peaks["source"] + " (burst bf16 GEMM)",
+                     "traffic": NCU_PREFILL_TRAFFIC_BYTES.get(w.name),
+                     "traffic_unit": "bytes per launch (ncu dram read + write)",
+                     "algorithmic_bytes": w.n_video * (2 * w.Hq * w.d * 2 + 2 * w.Hkv * w.d * 2 + w.Hq * 4)},
         "e2e": {"value": replicas.whole_job_rate(flops_layer, world, e2e_ms) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": KERNELS_PER_PASS * args.steps,

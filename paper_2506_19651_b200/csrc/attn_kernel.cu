@@ -395,6 +395,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         int ring_base = 0;  // ring position of this item's K(0)
 #ifdef PEVLM_PROFILE
         unsigned prof_busy = 0, prof_wait = 0, prof_t1 = 0, prof_t2 = static_cast<unsigned>(clock64()), prof_tiles = 0;
+        unsigned prof_ld = 0, prof_exp = 0;
 #endif
         for (int k = 0;; ++k) {
             const int w = next_item(k);
@@ -427,6 +428,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
                 tmem_wait_ld();
+#ifdef PEVLM_PROFILE
+                const unsigned prof_t_ld = static_cast<unsigned>(clock64());
+                prof_ld += prof_t_ld - prof_t1;
+#endif
                 if (need_mask) {
                     const int max_col = min(nvalid, my_limit - j0 + 1);
 #pragma unroll
@@ -492,6 +497,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     unpack_f32x2(add_f32x2(sm2[2], sm2[3]), b0, b1);
                     sum = (a0 + a1) + (b0 + b1);
                 }
+#ifdef PEVLM_PROFILE
+                const unsigned prof_t_exp = static_cast<unsigned>(clock64());
+                prof_exp += prof_t_exp - prof_t_ld;
+#endif
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(my_po);
@@ -516,6 +525,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             p.hdr->pad[8 + 8 * x] = static_cast<int32_t>(prof_busy >> 4);
             p.hdr->pad[9 + 8 * x] = static_cast<int32_t>(prof_wait >> 4);
             p.hdr->pad[10 + 8 * x] = static_cast<int32_t>(prof_tiles);
+            p.hdr->pad[11 + 8 * x] = static_cast<int32_t>(prof_ld >> 4);
+            p.hdr->pad[12 + 8 * x] = static_cast<int32_t>(prof_exp >> 4);
         }
 #endif
     } else {

@@ -100,7 +100,8 @@ def run_reference(args, w):
     if rank != 0:
         return
     q, k, v = inputs.make_qkv(w)
-    per_step = 8.0
+    # each step is a bounded sample; the whole run stays within about two minutes of oracle time
+    per_step = max(1.0, min(8.0, 120.0 / max(1, args.steps + args.warmup)))
     vals, secs = [], []
     last = None
     for i in range(args.warmup + args.steps):

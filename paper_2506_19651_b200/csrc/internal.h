@@ -67,6 +67,7 @@ struct RopeParams {
     int64_t first_token;
     int64_t n_tokens;
     int32_t Hq, Hkv;  // heads to process of each tensor (0 = skip tensor)
+    int32_t head_split;  // thread groups sharing one token's heads (set by launch_rope)
 };
 
 struct CopySegments {

@@ -22,7 +22,9 @@ __device__ __forceinline__ uint32_t f64_to_bf16_bits(double x) {
 // evaluates their 8 angles once in fp64 (sincos, kept in registers) and then walks over all
 // Hq + Hkv head vectors of that token, two 16-byte loads and two 16-byte stores per head.  The
 // d/16 threads of a token read 128 contiguous bytes per half head vector.  No shared memory,
-// no block-level synchronisation; CTAs stride over groups of 256 / (d/16) tokens.
+// no block-level synchronisation; CTAs stride over groups of 256 / (d/16) token slots.  For short
+// token ranges (the question block) the heads of a token are split over `head_split` such thread
+// groups, each evaluating the token's angles itself, so the launch still fills the machine.
 template <int D>
 __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constant__ RopeParams p) {
     constexpr int HALF = D / 2;
@@ -30,10 +32,13 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
     constexpr int TOK_PER_CTA = kRopeThreads / TPT;
     const int v = threadIdx.x % TPT;
     const int i0 = v * 8;
-    const int64_t n_groups = (p.n_tokens + TOK_PER_CTA - 1) / TOK_PER_CTA;
+    const int64_t n_slots = p.n_tokens * p.head_split;
+    const int64_t n_groups = (n_slots + TOK_PER_CTA - 1) / TOK_PER_CTA;
     for (int64_t grp = blockIdx.x; grp < n_groups; grp += gridDim.x) {
-        const int64_t tok = grp * TOK_PER_CTA + threadIdx.x / TPT;
-        if (tok >= p.n_tokens) continue;
+        const int64_t slot = grp * TOK_PER_CTA + threadIdx.x / TPT;
+        if (slot >= n_slots) continue;
+        const int64_t tok = slot / p.head_split;
+        const int h_first = static_cast<int>(slot % p.head_split);
         const int64_t pos = p.pos_ids ? static_cast<int64_t>(p.pos_ids[tok]) : p.first_token + tok;
         double cs[8], sn[8];
 #pragma unroll
@@ -42,7 +47,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
             sincos(ang, &sn[e], &cs[e]);
         }
         const int heads = p.Hq + p.Hkv;
-        for (int h = 0; h < heads; ++h) {
+        for (int h = h_first; h < heads; h += p.head_split) {
             const __nv_bfloat16* src;
             __nv_bfloat16* dst;
             if (h < p.Hq) {
@@ -84,13 +89,18 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
 cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream) {
     if (p.n_tokens <= 0 || p.Hq + p.Hkv == 0) return cudaSuccess;
     const int tok_per_cta = kRopeThreads / (head_dim / 16);
-    const int64_t groups = (p.n_tokens + tok_per_cta - 1) / tok_per_cta;
+    // enough thread groups for about two CTAs per SM, by splitting a token's heads if need be
+    RopeParams q = p;
+    q.head_split = 1;
+    while (q.head_split < 32 && q.head_split * 2 <= p.Hq + p.Hkv && p.n_tokens * q.head_split < 2 * 148 * tok_per_cta)
+        q.head_split *= 2;
+    const int64_t groups = (p.n_tokens * q.head_split + tok_per_cta - 1) / tok_per_cta;
     const int64_t cap = 148 * 8;  // whole waves of the 148 SMs; CTAs stride over the remaining groups
     const unsigned grid = static_cast<unsigned>(groups < cap ? groups : cap);
     if (head_dim == 128) {
-        rope_kernel<128><<<grid, kRopeThreads, 0, stream>>>(p);
+        rope_kernel<128><<<grid, kRopeThreads, 0, stream>>>(q);
     } else {
-        rope_kernel<64><<<grid, kRopeThreads, 0, stream>>>(p);
+        rope_kernel<64><<<grid, kRopeThreads, 0, stream>>>(q);
     }
     return cudaGetLastError();
 }

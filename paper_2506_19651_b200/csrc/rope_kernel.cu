@@ -12,10 +12,13 @@ constexpr int kRopeThreads = 256;
 __device__ __forceinline__ double bf16_bits_to_f64(uint32_t bits16) {
     return static_cast<double>(__uint_as_float(bits16 << 16));
 }
-// fp64 -> fp32 (round to nearest even) -> bf16 (round to nearest even): two roundings, in this order
-__device__ __forceinline__ uint32_t f64_to_bf16_bits(double x) {
-    const float f = __double2float_rn(x);
-    return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(f)));
+// fp64 -> fp32 (round to nearest even) -> bf16 (round to nearest even): two roundings, in this order;
+// the second one is done for two values at once by the packed conversion
+__device__ __forceinline__ uint32_t f64x2_to_bf16x2_bits(double lo, double hi) {
+    const float flo = __double2float_rn(lo), fhi = __double2float_rn(hi);
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(fhi), "f"(flo));
+    return r;
 }
 
 // A thread owns 8 rotation pairs (elements i0..i0+7 and i0+d/2..i0+d/2+7) of ONE token: it
@@ -66,19 +69,17 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
             uint32_t out_lo[4], out_hi[4];
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
-                uint32_t ra_bits[2], rb_bits[2];
+                double ra[2], rb[2];
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const double a = bf16_bits_to_f64((lo_w[w] >> (16 * e)) & 0xFFFFu);
                     const double b = bf16_bits_to_f64((hi_w[w] >> (16 * e)) & 0xFFFFu);
                     const double c = cs[2 * w + e], s = sn[2 * w + e];
-                    const double ra = __dsub_rn(__dmul_rn(a, c), __dmul_rn(b, s));
-                    const double rb = __dadd_rn(__dmul_rn(b, c), __dmul_rn(a, s));
-                    ra_bits[e] = f64_to_bf16_bits(ra);
-                    rb_bits[e] = f64_to_bf16_bits(rb);
+                    ra[e] = __dsub_rn(__dmul_rn(a, c), __dmul_rn(b, s));
+                    rb[e] = __dadd_rn(__dmul_rn(b, c), __dmul_rn(a, s));
                 }
-                out_lo[w] = ra_bits[0] | (ra_bits[1] << 16);
-                out_hi[w] = rb_bits[0] | (rb_bits[1] << 16);
+                out_lo[w] = f64x2_to_bf16x2_bits(ra[0], ra[1]);
+                out_hi[w] = f64x2_to_bf16x2_bits(rb[0], rb[1]);
             }
             *reinterpret_cast<uint4*>(dst + i0) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
             *reinterpret_cast<uint4*>(dst + i0 + HALF) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);

@@ -97,6 +97,29 @@ static float resolve_scale(const pevlm_shape_t* s) {
     return s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf(static_cast<float>(s->head_dim));
 }
 
+// ---- query tiles of one prefill segment (sink or context block) per kv head, shared by the launch and
+// the stats.  A segment of `len` tokens has ceil(len/128) tile positions; if the last one is ragged with
+// at most 64 rows, the tails of `tail_heads` q heads of the kv group share one 128-row tile.
+struct SegPlan {
+    int tiles, tail_rows, tail_heads, tail_tiles, full_tiles, entries, pairs;
+};
+
+static SegPlan plan_segment(int len, int G) {
+    SegPlan s;
+    s.tiles = (len + kTile - 1) / kTile;
+    s.tail_rows = 0; s.tail_heads = 0; s.tail_tiles = 0;
+    const int rem = len % kTile;
+    if (rem > 0 && rem <= kTile / 2 && G > 1) {
+        s.tail_rows = rem;
+        s.tail_heads = kTile / rem < G ? kTile / rem : G;
+        s.tail_tiles = (G + s.tail_heads - 1) / s.tail_heads;
+    }
+    s.full_tiles = s.tiles - (s.tail_tiles > 0 ? 1 : 0);
+    s.entries = s.tail_tiles + G * s.full_tiles;
+    s.pairs = (s.entries + 1) / 2;
+    return s;
+}
+
 // ---- question-attention decomposition (shared by the launch, the workspace size and the stats)
 struct QueryPlan {
     int tok_per_tile, q_tiles, total_kv_tiles, n_splits, tiles_per_split;
@@ -252,18 +275,25 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
     p.Hq = s->num_q_heads; p.Hkv = s->num_kv_heads; p.G = p.Hq / p.Hkv;
     p.tiles_sink = (p.S + kTile - 1) / kTile;
     p.tiles_block = p.N > 0 ? (p.B + kTile - 1) / kTile : 0;
-    p.pairs_block = (p.G * p.tiles_block + 1) / 2;
-    p.pairs_sink = (p.G * p.tiles_sink + 1) / 2;
+    const SegPlan pb = plan_segment(p.N > 0 ? p.B : 0, p.G), ps = plan_segment(p.S, p.G);
+    p.pairs_block = pb.pairs;
+    p.pairs_sink = ps.pairs;
+    p.tail_rows_block = pb.tail_rows; p.tail_heads_block = pb.tail_heads; p.tail_tiles_block = pb.tail_tiles;
+    p.tail_rows_sink = ps.tail_rows; p.tail_heads_sink = ps.tail_heads; p.tail_tiles_sink = ps.tail_tiles;
     p.items_block = p.N * p.Hkv * p.pairs_block;
     p.n_items = p.items_block + p.Hkv * p.pairs_sink;
-    p.q_box_rows = kTile;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
     p.hdr = static_cast<WorkspaceHeader*>(workspace);
     for (int b = 0; b < s->batch; ++b) {
         const int64_t qoff = static_cast<int64_t>(b) * nv * p.Hq * d, koff = static_cast<int64_t>(b) * nv * p.Hkv * d;
-        CUtensorMap tq, tk, tv;
-        if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q) + qoff, nv, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
+        CUtensorMap tq, tq_tb, tq_ts, tk, tv;
+        const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q) + qoff;
+        if ((rc = make_tmap(&tq, qb, nv, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
+        tq_tb = tq;
+        tq_ts = tq;
+        if (pb.tail_tiles > 0 && (rc = make_tmap(&tq_tb, qb, nv, p.Hq, d, pb.tail_heads, pb.tail_rows)) != PEVLM_OK) return rc;
+        if (ps.tail_tiles > 0 && (rc = make_tmap(&tq_ts, qb, nv, p.Hq, d, ps.tail_heads, ps.tail_rows)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         p.o = static_cast<__nv_bfloat16*>(o) + qoff;
@@ -272,7 +302,7 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
             e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
             if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
         }
-        e = launch_attn(p, d, tq, tk, tv, st);
+        e = launch_attn(p, d, tq, tq_tb, tq_ts, tk, tv, st);
         if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
     }
     return PEVLM_OK;
@@ -309,7 +339,6 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
     p.q_tiles = qp.q_tiles;
     p.n_splits = qp.n_splits;
     p.tiles_per_split = qp.tiles_per_split;
-    p.q_box_rows = p.G * p.tok_per_tile;
     p.n_items = p.Hkv * ((p.q_tiles + 1) / 2) * p.n_splits;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
@@ -329,7 +358,7 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
         if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        e = launch_attn(p, d, tq, tk, tv, st);
+        e = launch_attn(p, d, tq, tq, tq, tk, tv, st);
         if (e != cudaSuccess) return cuda_fail(e, "question attention launch");
         MergeParams m;
         m.Q = p.Q; m.Hq = p.Hq; m.d = d; m.n_splits = p.n_splits;
@@ -372,14 +401,27 @@ int pevlm_tile_stats(const pevlm_shape_t* s, int which, int64_t* tiles, double* 
     if (which == PEVLM_WS_PREFILL) {
         int64_t S = s->sink_len, B = s->num_blocks > 0 ? s->block_len : 0, N = s->num_blocks;
         if (s->mask_mode == PEVLM_MASK_FULL_CAUSAL) { S = 0; B = nv; N = nv > 0 ? 1 : 0; }
-        for (int64_t q0 = 0; q0 < S; q0 += kTile) add_range((q0 + kTile < S ? q0 + kTile : S));
+        const int G = s->num_q_heads / s->num_kv_heads;
+        // query tiles of one segment per kv head: G per full tile position, tail_tiles for a packed ragged tail
+        auto add_segment = [&](int64_t len, int64_t shared) {
+            const SegPlan sp = plan_segment(static_cast<int>(len), G);
+            for (int qt = 0; qt < sp.tiles; ++qt) {
+                const int64_t q0 = static_cast<int64_t>(qt) * kTile;
+                const int q_tiles = (sp.tail_tiles > 0 && qt == sp.tiles - 1) ? sp.tail_tiles : G;
+                const int64_t t0 = n_tiles; const double c0 = cols;
+                add_range(shared);
+                add_range(q0 + kTile < len ? q0 + kTile : len);
+                n_tiles = t0 + (n_tiles - t0) * q_tiles;
+                cols = c0 + (cols - c0) * q_tiles;
+            }
+        };
+        add_segment(S, 0);
         const int64_t t0 = n_tiles; const double c0 = cols;
-        for (int64_t q0 = 0; q0 < B; q0 += kTile) { add_range(S); add_range((q0 + kTile < B ? q0 + kTile : B)); }
-        // the block part repeats for each of the N blocks
-        n_tiles = t0 + (n_tiles - t0) * N;
+        add_segment(B, S);
+        n_tiles = t0 + (n_tiles - t0) * N;   // the block part repeats for each of the N blocks
         cols = c0 + (cols - c0) * static_cast<double>(N);
-        n_tiles *= s->num_q_heads;
-        cols *= s->num_q_heads;
+        n_tiles *= s->num_kv_heads;
+        cols *= s->num_kv_heads;
     } else if (which == PEVLM_WS_QUERY) {
         const QueryPlan qp = plan_query(s);
         for (int qt = 0; qt < qp.q_tiles; ++qt) {

@@ -16,7 +16,7 @@
 //   warp 13     work scheduler and TMA producer: takes the next work item from a global
 //               counter, publishes it to the other roles, loads its two Q tiles, then streams
 //               K/V tiles through a 4-slot ring that runs on across items
-// The kernel is persistent (one CTA per SM): while the correction warps write out item k, the
+// The kernel is persistent (one CTA per SM): while the epilogue warps write out item k, the
 // producer, the MMA warp and the softmax warps already work on item k+1.
 // TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
 // Every wait is bounded; an expired wait records PEVLM_ETIMEOUT and the CTA still runs to its
@@ -64,12 +64,16 @@ size_t attn_smem_bytes(int head_dim) {
     return 1024 + (head_dim == 128 ? AttnSmem<128>::kTotal : AttnSmem<64>::kTotal);
 }
 
+// One query tile.  Row r of the tile is token q_tok0 + r / row_div, head q_head0 + r % row_div; it
+// exists iff r / row_div < ntok and r % row_div < nheads.  Full prefill tiles have row_div = 1; the
+// ragged last tile of a segment packs the tails of several q heads of the kv group (row_div heads,
+// ntok = the tail's rows); question tiles pack all G heads of the group.
 struct QSlot {
     int valid;
-    int q_tok0, q_head0, rows_valid, limit0, b_end, nt;
+    int q_tok0, q_head0, row_div, ntok, nheads, qmap, box_rows, limit0, b_end, nt;
 };
 struct WorkItem {
-    int kv_head, row_div, a_end, b_start, na, split;
+    int kv_head, a_end, b_start, na, split;
     QSlot s[2];
 };
 
@@ -78,8 +82,7 @@ __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
 __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem& it) {
     it.split = 0;
     if (p.mode == 0) {
-        it.row_div = 1;
-        int seg_start, seg_len, tiles, pi, g;
+        int seg_start, seg_len, tiles, pi, g, tail_rows, tail_heads, tail_tiles, qmap_tail;
         if (w < p.items_block) {
             const int combo = w / p.pairs_block;
             pi = w % p.pairs_block;
@@ -88,6 +91,8 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             seg_start = p.S + blk * p.B;
             seg_len = p.B;
             tiles = p.tiles_block;
+            tail_rows = p.tail_rows_block; tail_heads = p.tail_heads_block; tail_tiles = p.tail_tiles_block;
+            qmap_tail = 1;
             it.a_end = p.S;
         } else {
             const int w2 = w - p.items_block;
@@ -96,20 +101,42 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             seg_start = 0;
             seg_len = p.S;
             tiles = p.tiles_sink;
+            tail_rows = p.tail_rows_sink; tail_heads = p.tail_heads_sink; tail_tiles = p.tail_tiles_sink;
+            qmap_tail = 2;
             it.a_end = 0;
         }
         it.kv_head = g;
         it.b_start = seg_start;
         it.na = cdiv(it.a_end, kTile);
+        // entries of this (segment, kv head), heaviest first: the packed tail tiles (last tile position of
+        // the segment, tail_heads q heads each), then (tile position, q head) for the full positions
+        const int full_tiles = tiles - (tail_tiles > 0 ? 1 : 0);
+        const int entries = tail_tiles + p.G * full_tiles;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
             const int e = 2 * pi + x;
             QSlot& s = it.s[x];
-            s.valid = e < p.G * tiles;
-            const int qt = tiles - 1 - e / p.G;  // heaviest query tiles first
+            s.valid = e < entries;
+            int qt;
+            if (e < tail_tiles) {
+                qt = tiles - 1;
+                s.q_head0 = g * p.G + e * tail_heads;
+                s.row_div = tail_heads;
+                s.ntok = tail_rows;
+                s.nheads = min(tail_heads, p.G - e * tail_heads);
+                s.qmap = qmap_tail;
+                s.box_rows = tail_heads * tail_rows;
+            } else {
+                const int e2 = e - tail_tiles;
+                qt = full_tiles - 1 - e2 / p.G;
+                s.q_head0 = g * p.G + e2 % p.G;
+                s.row_div = 1;
+                s.ntok = min(kTile, seg_len - qt * kTile);
+                s.nheads = 1;
+                s.qmap = 0;
+                s.box_rows = kTile;
+            }
             s.q_tok0 = seg_start + qt * kTile;
-            s.q_head0 = g * p.G + e % p.G;
-            s.rows_valid = min(kTile, seg_len - qt * kTile);
             s.limit0 = s.q_tok0;
             s.b_end = min(s.q_tok0 + kTile, seg_start + seg_len);
             s.nt = s.valid ? it.na + cdiv(s.b_end - it.b_start, kTile) : 0;
@@ -121,7 +148,6 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
         const int pi = rest % q_pairs;
         const int g = rest / q_pairs;
         it.kv_head = g;
-        it.row_div = p.G;
         it.a_end = 0;
         it.na = 0;
         const int split_lo = it.split * p.tiles_per_split * kTile;
@@ -136,7 +162,11 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             const int ntok = max(0, min(p.tok_per_tile, p.Q - tok0));
             s.q_tok0 = tok0;
             s.q_head0 = g * p.G;
-            s.rows_valid = ntok * p.G;
+            s.row_div = p.G;
+            s.ntok = ntok;
+            s.nheads = p.G;
+            s.qmap = 0;
+            s.box_rows = p.G * p.tok_per_tile;
             s.limit0 = p.n_video + tok0;
             const int kv_end = p.n_video + tok0 + ntok;  // keys past the last row's limit are never visible
             s.b_end = min(kv_end, split_hi);
@@ -148,7 +178,8 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap tmap_q,
-               const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+            const __grid_constant__ CUtensorMap tmap_q_tail_block, const __grid_constant__ CUtensorMap tmap_q_tail_sink,
+            const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
     using L = AttnSmem<D>;
     constexpr int NP = L::kPanels;
     extern __shared__ uint8_t smem_raw[];
@@ -192,6 +223,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         }
         fence_mbar_init();
         tma_prefetch_desc(&tmap_q);
+        tma_prefetch_desc(&tmap_q_tail_block);
+        tma_prefetch_desc(&tmap_q_tail_sink);
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
     }
@@ -241,9 +274,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 for (int x = 0; x < 2; ++x) {
                     if (it.s[x].nt == 0) continue;
                     if (q_loads[x] > 0) wait(bar_q_free + 8 * x, (q_loads[x] - 1) & 1, kWaitQFree);
-                    mbar_arrive_expect_tx(bar_q_full + 8 * x, static_cast<uint32_t>(NP * p.q_box_rows * 128));
+                    mbar_arrive_expect_tx(bar_q_full + 8 * x, static_cast<uint32_t>(NP * it.s[x].box_rows * 128));
+                    const CUtensorMap* qmap = it.s[x].qmap == 0 ? &tmap_q : it.s[x].qmap == 1 ? &tmap_q_tail_block : &tmap_q_tail_sink;
                     for (int h = 0; h < NP; ++h)
-                        tma_load_3d(smem_base + (x ? L::kQ1 : L::kQ0) + h * L::kPanelBytes, &tmap_q, h * 64,
+                        tma_load_3d(smem_base + (x ? L::kQ1 : L::kQ0) + h * L::kPanelBytes, qmap, h * 64,
                                     it.s[x].q_head0, it.s[x].q_tok0, bar_q_full + 8 * x);
                     ++q_loads[x];
                 }
@@ -410,7 +444,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
             const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
             const int na = it.na, a_end = it.a_end, b_start = it.b_start;
-            const int my_limit = limit0 + row / it.row_div;
+            const int my_limit = limit0 + row / (x ? it.s[1].row_div : it.s[0].row_div);
             float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
             float l_run = 0.f;
             for (int j = 0; j < nt; ++j, ++cnt) {
@@ -544,9 +578,9 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             for (int x = 0; x < 2; ++x) {
                 const QSlot& s = it.s[x];
                 if (!s.valid) continue;
-                const bool row_ok = row < s.rows_valid;
-                const int tok = s.q_tok0 + row / it.row_div;
-                const int head = s.q_head0 + row % it.row_div;
+                const bool row_ok = (row / s.row_div < s.ntok) && (row % s.row_div < s.nheads);
+                const int tok = s.q_tok0 + row / s.row_div;
+                const int head = s.q_head0 + row % s.row_div;
                 if (s.nt == 0) {
                     // question-mode slot with no visible key in this CTA's key range: neutral partial
                     if (p.mode == 1 && row_ok) {
@@ -616,8 +650,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     }
 }
 
-cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
-                           const CUtensorMap& tv, cudaStream_t stream) {
+cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tq_tail_block,
+                        const CUtensorMap& tq_tail_sink, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
     const size_t smem = attn_smem_bytes(head_dim);
     int dev = 0, sms = 0;
@@ -629,11 +663,11 @@ cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<128><<<grid, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_kernel<128><<<grid, kAttnThreads, smem, stream>>>(p, tq, tq_tail_block, tq_tail_sink, tk, tv);
     } else {
         e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<64><<<grid, kAttnThreads, smem, stream>>>(p, tq, tk, tv);
+        attn_kernel<64><<<grid, kAttnThreads, smem, stream>>>(p, tq, tq_tail_block, tq_tail_sink, tk, tv);
     }
     return cudaGetLastError();
 }

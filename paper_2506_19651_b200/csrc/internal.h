@@ -35,7 +35,10 @@ struct AttnParams {
     int32_t pairs_sink;     // ceil(G * tiles_sink / 2) query-tile pairs per kv head
     int32_t items_block;    // N * Hkv * pairs_block work items over the context blocks
     int32_t n_items;        // all work items of the launch
-    int32_t q_box_rows;     // rows the Q TMA box brings in (128 prefill, G * tok_per_tile question)
+    // ragged last query tile of a segment (len % 128 rows): the tails of tail_heads q heads of one kv
+    // group are packed into one 128-row tile, tail_tiles such tiles per (segment, kv head); 0 = no packing
+    int32_t tail_rows_block, tail_heads_block, tail_tiles_block;
+    int32_t tail_rows_sink, tail_heads_sink, tail_tiles_sink;
     int32_t tok_per_tile;   // mode 1: question tokens per query tile = 128 / G
     int32_t q_tiles;        // mode 1: ceil(Q / tok_per_tile)
     int32_t n_splits;       // mode 1
@@ -79,8 +82,8 @@ struct CopySegments {
 
 cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream);
 cudaError_t launch_copy_segments(const CopySegments& s, cudaStream_t stream);
-cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tk,
-                        const CUtensorMap& tv, cudaStream_t stream);
+cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tq_tail_block,
+                        const CUtensorMap& tq_tail_sink, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 size_t attn_smem_bytes(int head_dim);
 // error reporting shared by the host-side translation units: both record a text that

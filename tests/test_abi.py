@@ -61,6 +61,21 @@ def test_tile_stats_closed_form(lib):
     assert st.flops == 4.0 * 128 * 128 * (cols_tri + 7 * 784 + cols_tri)
 
 
+def test_tile_stats_packed_ragged_tails(lib):
+    # 1568 = 12 * 128 + 32: the 32-row tails of 4 of the 7 q heads of a kv group share one query tile,
+    # so a (segment, kv head) has 12 * 7 full tiles and ceil(7 / 4) = 2 tail tiles
+    S = B = 1568
+    N, Hq, Hkv = 2, 28, 4
+    st = pb.pevlm_tile_stats(pb.make_shape(S, B, N, 0, Hq, Hkv, 128), pb.WS_PREFILL)
+    G = Hq // Hkv
+    sink_tiles = sum((qt + 1) * G for qt in range(12)) + 13 * 2          # key tiles per query tile: qt + 1
+    block_tiles = sum((13 + qt + 1) * G for qt in range(12)) + (13 + 13) * 2
+    assert st.tiles == Hkv * (sink_tiles + N * block_tiles)
+    # more than 64 tail rows: no packing (every head keeps its own ragged tile)
+    st2 = pb.pevlm_tile_stats(pb.make_shape(200, 200, 1, 0, 4, 2, 128), pb.WS_PREFILL)
+    assert st2.tiles == 4 * ((1 + 2) + (2 + 1) + (2 + 2))
+
+
 def test_argument_errors_before_launch(lib):
     good = pb.make_shape(64, 128, 4, 32, 4, 2, 64)
     ws = C.c_void_p(256 * 4)

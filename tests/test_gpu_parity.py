@@ -212,3 +212,45 @@ def test_full_causal_mode_full_size_sampled_rows():
     errs, _, _ = check_against_oracle(w, q, k, v, res, rows[rows < w.n_video], full_causal=True)
     for key, e in errs.items():
         assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)
+
+
+# ---------------------------------------------------------------- position and mask variants (no new kernels)
+
+def test_reused_positions_per_block_variant():
+    """The comparison the paper draws in Sec. 3.2.2 / Sec. 5.1: positions restarting in every block (what
+    prior parallel-encoding methods do) instead of sequential ones.  Only the position ids change."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(96, 160, 3, 0, 4, 2, 128)
+    q, k, v = inputs.make_qkv(w)
+    t = np.arange(w.L)
+    pos = np.where(t < w.S, t, w.S + (t - w.S) % w.B).astype(np.int32)      # every block restarts after the sink
+    s = gpu_shape(w)
+    qd, kd = to_dev(q), to_dev(k)
+    pb.pevlm_rope_qk(s, qd, kd, qd, kd, 0, w.L, torch.from_numpy(pos).cuda())
+    o = torch.empty_like(qd)
+    lse = torch.empty((w.Hq, w.L), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device="cuda")
+    pb.pevlm_parallel_prefill_attn(s, qd, kd, to_dev(v), o, lse, ws)
+    torch.cuda.synchronize()
+    qr, kr = oracle.rope(q, w.theta, pos=pos.astype(np.int64)), oracle.rope(k, w.theta, pos=pos.astype(np.int64))
+    np.testing.assert_array_equal(to_bits(qd), qr)
+    o_ref, lse_ref = oracle.attn_rows(oracle.make_shape(w.S, w.B, w.N, 0, w.Hq, w.Hkv, w.d), qr, kr, v, np.arange(w.L))
+    assert np.abs(bits_to_f64(to_bits(o)) - o_ref).max() <= O_TOL
+    assert np.abs(lse.double().cpu().numpy().T - lse_ref).max() <= LSE_TOL
+    # and it differs from the sequential-position result on the context rows (the method's point)
+    o_seq, _ = oracle.attn_rows(oracle.make_shape(w.S, w.B, w.N, 0, w.Hq, w.Hkv, w.d), oracle.rope(q, w.theta),
+                                oracle.rope(k, w.theta), v, np.arange(w.S + w.B, w.L))
+    assert np.abs(o_seq - o_ref[w.S + w.B:]).max() > 1e-2
+
+
+@pytest.mark.parametrize("Q", [1, 2, 5])
+def test_decode_sized_question_blocks(Q):
+    """A few new rows against the assembled cache (the step after prefill): the question attention with
+    1 to 5 query tokens, i.e. 7 to 35 rows of a 128-row tile."""
+    w = wl(300, 260, 3, Q, 28, 4, 128, outliers=True)
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v)
+    errs, _, _ = check_against_oracle(w, q, k, v, res, np.arange(w.n_video, w.L))
+    for key, e in errs.items():
+        assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)

@@ -69,6 +69,20 @@ def rope(x_bits, theta: float, pos=None, first_pos: int = 0, want_f64: bool = Fa
     return (out, f64) if want_f64 else out
 
 
+def rope_mrope(x_bits, theta: float, pos3, sections, want_f64: bool = False):
+    """Multimodal RoPE: pos3 [3, n] (temporal, height, width), sections = pairs per component."""
+    x = _u16(x_bits)
+    n, heads, d = x.shape
+    pos3 = np.ascontiguousarray(pos3, dtype=np.int64)
+    assert pos3.shape == (3, n) and sum(sections) == d // 2
+    sec = np.ascontiguousarray(sections, dtype=np.int32)
+    out = np.empty_like(x)
+    f64 = np.empty(x.shape, dtype=np.float64) if want_f64 else None
+    lib().oracle_rope_mrope(_p(x), C.c_int64(n), C.c_int32(heads), C.c_int32(d), C.c_double(theta),
+                            _p(pos3), _p(sec), _p(out), _p(f64))
+    return (out, f64) if want_f64 else out
+
+
 def attn_rows(sh: Shape, q_bits, k_bits, v_bits, rows, scale: float = 0.0, key_lo: int = -1, key_hi: int = -1):
     """Rows of masked softmax attention.  Returns (o [n,Hq,d] fp64, lse [n,Hq] fp64)."""
     q, k, v = _u16(q_bits), _u16(k_bits), _u16(v_bits)

@@ -126,6 +126,41 @@ void oracle_rope(const uint16_t* x, int64_t n_tokens, int32_t heads, int32_t d, 
 }
 
 /*
+ * Multimodal RoPE (the position embedding of the Qwen2-VL family the paper evaluates, Sec. 3.1: positions
+ * carry temporal and spatial components).  Each token has three position components pos3[c][t], c = 0
+ * temporal, 1 height, 2 width; rotary pair i uses component 0 for i < sec[0], component 1 for the next
+ * sec[1] pairs and component 2 for the rest (sec[0] + sec[1] + sec[2] = d/2).  Everything else as
+ * oracle_rope: rotate-half pairing, fp64, one rounding to bf16.  With three equal components it is
+ * oracle_rope.
+ */
+void oracle_rope_mrope(const uint16_t* x, int64_t n_tokens, int32_t heads, int32_t d, double theta,
+                       const int64_t* pos3, const int32_t* sec, uint16_t* out_bits, double* out_f64) {
+    int32_t half = d / 2;
+    double* inv_freq = (double*)malloc(sizeof(double) * (size_t)half);
+    for (int32_t i = 0; i < half; ++i) inv_freq[i] = pow(theta, -2.0 * (double)i / (double)d);
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < n_tokens; ++t) {
+        for (int32_t h = 0; h < heads; ++h) {
+            const uint16_t* xr = x + ((size_t)t * heads + h) * d;
+            for (int32_t i = 0; i < half; ++i) {
+                int c = (i < sec[0]) ? 0 : (i < sec[0] + sec[1]) ? 1 : 2;
+                double p = (double)pos3[(size_t)c * n_tokens + t];
+                double ang = p * inv_freq[i];
+                double co = cos(ang), si = sin(ang);
+                double a = bf16_to_f64(xr[i]);
+                double b = bf16_to_f64(xr[i + half]);
+                double ra = a * co - b * si;
+                double rb = b * co + a * si;
+                size_t o = ((size_t)t * heads + h) * d;
+                if (out_f64) { out_f64[o + i] = ra; out_f64[o + i + half] = rb; }
+                if (out_bits) { out_bits[o + i] = f64_to_bf16(ra); out_bits[o + i + half] = f64_to_bf16(rb); }
+            }
+        }
+    }
+    free(inv_freq);
+}
+
+/*
  * Masked softmax attention (Eq. 1 under the masks of Eq. 3-5) for a list of query rows,
  * all q heads.  q: [L,Hq,d], k,v: [L,Hkv,d], bf16 bits, q and k already roped.
  * rows[n_rows]: global token indices.  o: [n_rows,Hq,d] fp64, lse: [n_rows,Hq] fp64.

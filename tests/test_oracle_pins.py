@@ -283,6 +283,23 @@ def test_p7_huge_theta_rotates_only_first_pair():
     assert np.abs(f64[..., [0, 4]] - x[..., [0, 4]]).max() > 1e-3
 
 
+def test_p7_mrope_reduces_to_rope_and_uses_the_right_component():
+    # three equal components: bit-identical to plain RoPE at those positions
+    w = inputs.Workload("t", 9, 1, 0, 0, 2, 2, 16, 1e6, False, 4)
+    q, _, _ = inputs.make_qkv(w)
+    pos = np.array([0, 5, 77, 1234, 70000, 3, 3, 9, 12], dtype=np.int64)
+    np.testing.assert_array_equal(api.rope_mrope(q, 1e6, np.stack([pos, pos, pos]), [3, 3, 2]), api.rope(q, 1e6, pos=pos))
+    # d = 4, sections [1, 1, 0]: pair (0,2) turns by the temporal position, pair (1,3) by the height position
+    # times theta^(-1/2) = 0.01; hand values with cos(1), sin(1)
+    x = _bits([1.0, 1.0, 0.0, 0.0]).reshape(1, 1, 4)
+    _, f64 = api.rope_mrope(x, 1e4, np.array([[1], [100], [555]]), [1, 1, 0], want_f64=True)
+    np.testing.assert_allclose(f64[0, 0], [COS1, COS1, SIN1, SIN1], rtol=0, atol=1e-15)
+    # sections [0, 1, 1]: pair 0 by height (angle 100: not cos 1), pair 1 by width 100 * 0.01 = 1
+    _, f64 = api.rope_mrope(x, 1e4, np.array([[1], [100], [100]]), [0, 1, 1], want_f64=True)
+    np.testing.assert_allclose(f64[0, 0, [1, 3]], [COS1, SIN1], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(f64[0, 0, [0, 2]], [math.cos(100.0), math.sin(100.0)], rtol=0, atol=1e-14)
+
+
 # ---- P8: LSE merge of key-range partials reproduces the unsplit result ---------------
 
 @pytest.mark.parametrize("cuts", [[0, 9, 20, 31], [0, 31], [0, 0, 5, 5, 31], [0, 1, 2, 30, 31, 40]])

@@ -87,6 +87,20 @@ int pevlm_rope_qk(const pevlm_shape_t* shape, const void* q_in, const void* k_in
                   void* stream);
 
 /*
+ * Multimodal RoPE, the position embedding of the Qwen2-VL family the paper evaluates ("their position
+ * embeddings also incorporate spatio-temporal information", Sec. 3.1): every token has three position
+ * components, pos_ids3 = device int32 [3, n_tokens] (temporal, height, width).  Rotary pair i < d/2 takes
+ * its position from component 0 for i < sections[0], from component 1 for the next sections[1] pairs and
+ * from component 2 for the last sections[2] (host int32[3], sum = d/2; the split itself is the model's,
+ * not the paper's, e.g. {16, 24, 24} at d = 128).  Sequential positions in the sense of Sec. 3.2.2 means
+ * the ids are those of the unpartitioned stream.  Everything else as pevlm_rope_qk (fp64 evaluation, one
+ * rounding, in place or out of place, NULL pairs skipped); batch applies to pos_ids3 as [batch, 3, n_tokens].
+ */
+int pevlm_rope_qk_mrope(const pevlm_shape_t* shape, const void* q_in, const void* k_in, void* q_out,
+                        void* k_out, int64_t n_tokens, const int32_t* pos_ids3, const int32_t* sections,
+                        void* stream);
+
+/*
  * Prefill attention of the video tokens [Eq. 3, Eq. 4]: rows [0, S + N*B).
  *   q [S+N*B, Hq, d], k, v [S+N*B, Hkv, d]  (q, k already roped), read only
  *   o [S+N*B, Hq, d] bf16, lse [Hq, S+N*B] fp32 (may be NULL), written

@@ -21,7 +21,7 @@ WS_PREFILL, WS_QUERY = 0, 1
 
 NOALLOC_SCRATCH_BYTES = 32 << 20
 
-EXPORTS = ["pevlm_rope_qk", "pevlm_parallel_prefill_attn", "pevlm_assemble_kv", "pevlm_query_attn",
+EXPORTS = ["pevlm_rope_qk", "pevlm_rope_qk_mrope", "pevlm_parallel_prefill_attn", "pevlm_assemble_kv", "pevlm_query_attn",
            "pevlm_query_attn_noalloc",
            "pevlm_workspace_bytes", "pevlm_read_status", "pevlm_tile_stats", "pevlm_strerror",
            "pevlm_last_cuda_error"]
@@ -67,6 +67,8 @@ def lib():
         l = C.CDLL(LIB_PATH)
         vp, sp = C.c_void_p, C.POINTER(Shape)
         l.pevlm_rope_qk.argtypes = [sp, vp, vp, vp, vp, C.c_int64, C.c_int64, vp, vp]
+        l.pevlm_rope_qk_mrope.argtypes = [sp, vp, vp, vp, vp, C.c_int64, vp, C.POINTER(C.c_int32), vp]
+        l.pevlm_rope_qk_mrope.restype = C.c_int
         l.pevlm_parallel_prefill_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         l.pevlm_assemble_kv.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp]
         l.pevlm_query_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
@@ -107,6 +109,12 @@ def pevlm_workspace_bytes(shape: Shape, which: int) -> int:
 def pevlm_rope_qk(shape: Shape, q_in, k_in, q_out, k_out, first_token: int, n_tokens: int, pos_ids=None):
     _check(lib().pevlm_rope_qk(C.byref(shape), _ptr(q_in), _ptr(k_in), _ptr(q_out), _ptr(k_out),
                                first_token, n_tokens, _ptr(pos_ids), _stream()), "pevlm_rope_qk")
+
+
+def pevlm_rope_qk_mrope(shape: Shape, q_in, k_in, q_out, k_out, n_tokens: int, pos_ids3, sections):
+    sec = (C.c_int32 * 3)(*sections)
+    _check(lib().pevlm_rope_qk_mrope(C.byref(shape), _ptr(q_in), _ptr(k_in), _ptr(q_out), _ptr(k_out),
+                                     n_tokens, _ptr(pos_ids3), sec, _stream()), "pevlm_rope_qk_mrope")
 
 
 def pevlm_parallel_prefill_attn(shape: Shape, q, k, v, o, lse, workspace):

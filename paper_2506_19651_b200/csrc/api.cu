@@ -180,8 +180,9 @@ size_t pevlm_workspace_bytes(const pevlm_shape_t* s, int which) {
     return 0;
 }
 
-int pevlm_rope_qk(const pevlm_shape_t* s, const void* q_in, const void* k_in, void* q_out, void* k_out,
-                  int64_t first_token, int64_t n_tokens, const int32_t* pos_ids, void* stream) {
+static int rope_common(const pevlm_shape_t* s, const void* q_in, const void* k_in, void* q_out, void* k_out,
+                       int64_t first_token, int64_t n_tokens, const int32_t* pos_ids, const int32_t* pos3,
+                       const int32_t* sections, void* stream) {
     int rc = check_shape(s);
     if (rc != PEVLM_OK) return rc;
     if (n_tokens < 0 || first_token < 0 || first_token + n_tokens > (1ll << 31)) return PEVLM_EINVAL;
@@ -189,15 +190,23 @@ int pevlm_rope_qk(const pevlm_shape_t* s, const void* q_in, const void* k_in, vo
     if (!q_in && !k_in) return PEVLM_EINVAL;
     if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(q_out) || !aligned16(k_out)) return PEVLM_EALIGN;
     if (pos_ids && (reinterpret_cast<uintptr_t>(pos_ids) & 3u)) return PEVLM_EALIGN;
+    if (pos3 && (reinterpret_cast<uintptr_t>(pos3) & 3u)) return PEVLM_EALIGN;
+    const int d = s->head_dim;
+    if (sections) {
+        if (sections[0] < 0 || sections[1] < 0 || sections[2] < 0 || sections[0] + sections[1] + sections[2] != d / 2)
+            return PEVLM_EINVAL;
+    }
     if (n_tokens == 0) return PEVLM_OK;
     RopeParams p;
-    const int d = s->head_dim;
     for (int i = 0; i < d / 2; ++i) p.inv_freq[i] = pow(static_cast<double>(s->rope_theta), -2.0 * i / d);
     for (int i = d / 2; i < 64; ++i) p.inv_freq[i] = 0.0;
     p.first_token = first_token;
     p.n_tokens = n_tokens;
     p.Hq = q_in ? s->num_q_heads : 0;
     p.Hkv = k_in ? s->num_kv_heads : 0;
+    p.head_split = 1;
+    p.sec_end0 = sections ? sections[0] : 0;
+    p.sec_end1 = sections ? sections[0] + sections[1] : 0;
     for (int b = 0; b < s->batch; ++b) {
         const int64_t qo = static_cast<int64_t>(b) * n_tokens * s->num_q_heads * d;
         const int64_t ko = static_cast<int64_t>(b) * n_tokens * s->num_kv_heads * d;
@@ -206,10 +215,22 @@ int pevlm_rope_qk(const pevlm_shape_t* s, const void* q_in, const void* k_in, vo
         p.k_in = k_in ? static_cast<const __nv_bfloat16*>(k_in) + ko : nullptr;
         p.k_out = k_out ? static_cast<__nv_bfloat16*>(k_out) + ko : nullptr;
         p.pos_ids = pos_ids ? pos_ids + static_cast<int64_t>(b) * n_tokens : nullptr;
+        p.pos3 = pos3 ? pos3 + static_cast<int64_t>(b) * 3 * n_tokens : nullptr;
         cudaError_t e = launch_rope(p, d, static_cast<cudaStream_t>(stream));
         if (e != cudaSuccess) return cuda_fail(e, "rope launch");
     }
     return PEVLM_OK;
+}
+
+int pevlm_rope_qk(const pevlm_shape_t* s, const void* q_in, const void* k_in, void* q_out, void* k_out,
+                  int64_t first_token, int64_t n_tokens, const int32_t* pos_ids, void* stream) {
+    return rope_common(s, q_in, k_in, q_out, k_out, first_token, n_tokens, pos_ids, nullptr, nullptr, stream);
+}
+
+int pevlm_rope_qk_mrope(const pevlm_shape_t* s, const void* q_in, const void* k_in, void* q_out, void* k_out,
+                        int64_t n_tokens, const int32_t* pos_ids3, const int32_t* sections, void* stream) {
+    if (!pos_ids3 || !sections) return PEVLM_EINVAL;
+    return rope_common(s, q_in, k_in, q_out, k_out, 0, n_tokens, nullptr, pos_ids3, sections, stream);
 }
 
 int pevlm_assemble_kv(const pevlm_shape_t* s, const void* k_video, const void* v_video, const void* k_question,

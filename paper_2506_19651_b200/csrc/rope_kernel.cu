@@ -46,7 +46,13 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
         double cs[8], sn[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const double ang = __dmul_rn(static_cast<double>(pos), p.inv_freq[i0 + e]);
+            int64_t pe = pos;
+            if (p.pos3) {  // multimodal: the pair's section picks the temporal, height or width position
+                const int i = i0 + e;
+                const int comp = i < p.sec_end0 ? 0 : i < p.sec_end1 ? 1 : 2;
+                pe = static_cast<int64_t>(p.pos3[comp * p.n_tokens + tok]);
+            }
+            const double ang = __dmul_rn(static_cast<double>(pe), p.inv_freq[i0 + e]);
             sincos(ang, &sn[e], &cs[e]);
         }
         const int heads = p.Hq + p.Hkv;

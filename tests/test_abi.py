@@ -99,6 +99,11 @@ def test_argument_errors_before_launch(lib):
     assert lib.pevlm_rope_qk(C.byref(good), p16, None, None, None, 0, 8, None, None) == pb.PEVLM_EINVAL
     assert lib.pevlm_rope_qk(C.byref(good), odd, None, odd, None, 0, 8, None, None) == pb.PEVLM_EALIGN
     assert lib.pevlm_rope_qk(C.byref(good), p16, None, p16, None, -1, 8, None, None) == pb.PEVLM_EINVAL
+    sec_bad = (C.c_int32 * 3)(16, 24, 23)
+    sec_ok = (C.c_int32 * 3)(8, 12, 12)
+    assert lib.pevlm_rope_qk_mrope(C.byref(good), p16, None, p16, None, 8, p16, sec_bad, None) == pb.PEVLM_EINVAL
+    assert lib.pevlm_rope_qk_mrope(C.byref(good), p16, None, p16, None, 8, None, sec_ok, None) == pb.PEVLM_EINVAL
+    assert lib.pevlm_rope_qk_mrope(C.byref(good), odd, None, odd, None, 8, p16, sec_ok, None) == pb.PEVLM_EALIGN
     assert lib.pevlm_assemble_kv(C.byref(good), p16, None, None, None, None, None, None) == pb.PEVLM_EINVAL
     assert lib.pevlm_query_attn(C.byref(good), p16, p16, p16, p16, None, ws, 16, None) == pb.PEVLM_EWORKSPACE
 

@@ -254,3 +254,25 @@ def test_decode_sized_question_blocks(Q):
     errs, _, _ = check_against_oracle(w, q, k, v, res, np.arange(w.n_video, w.L))
     for key, e in errs.items():
         assert e <= (LSE_TOL if key.startswith("lse") else O_TOL), (key, e, errs)
+
+
+# ---------------------------------------------------------------- multimodal RoPE (three position components)
+
+@pytest.mark.parametrize("n,Hq,Hkv,d,sections", [(300, 28, 4, 128, (16, 24, 24)), (77, 4, 2, 64, (8, 12, 12)), (5, 2, 2, 128, (64, 0, 0))])
+def test_mrope_bit_exact(n, Hq, Hkv, d, sections):
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(n, 1, 0, 0, Hq, Hkv, d, 1e6)
+    q, k, _ = inputs.make_qkv(w)
+    rng = np.random.default_rng(5)
+    # a video-like id grid: temporal id per frame, height/width ids inside the frame, all offset by a text prefix
+    t_id = 40 + np.arange(n) // 16
+    pos3 = np.stack([t_id, 40 + (np.arange(n) % 16) // 4, 40 + np.arange(n) % 4]).astype(np.int32)
+    pos3[:, :3] = rng.integers(0, 70000, size=(1, 3))            # text tokens: equal components, large values
+    s = gpu_shape(w)
+    qd, kd = to_dev(q), to_dev(k)
+    qo, ko = torch.empty_like(qd), torch.empty_like(kd)
+    pb.pevlm_rope_qk_mrope(s, qd, kd, qo, ko, n, torch.from_numpy(pos3).cuda(), sections)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_bits(qo), oracle.rope_mrope(q, 1e6, pos3, sections))
+    np.testing.assert_array_equal(to_bits(ko), oracle.rope_mrope(k, 1e6, pos3, sections))

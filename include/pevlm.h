@@ -113,6 +113,25 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* shape, const void* q, const
                                 size_t workspace_bytes, void* stream);
 
 /*
+ * Attention of a range of context blocks against a resident cache [Eq. 4 for those blocks alone]: the
+ * num_blocks blocks of block_len tokens whose roped K and V sit at rows [first_key_row, first_key_row + N*B)
+ * of k_cache / v_cache [cache_rows, Hkv, d]; rows [0, S) of the cache are the sink.  Each block sees the
+ * sink and itself causally, exactly as in pevlm_parallel_prefill_attn; the sink rows are not recomputed.
+ *   q_blocks [N*B, Hq, d] roped, o [N*B, Hq, d], lse [Hq, N*B] (may be NULL): the block rows only.
+ * Because blocks do not attend to one another (Sec. 1), this one call serves (i) a video whose length is
+ * not a multiple of the block length (Sec. 3.2.1 partitions uniformly and is silent on a remainder: the
+ * remainder is taken as one shorter last block, run with block_len = its length), (ii) a streaming window
+ * that encodes one new block against the fixed sink into any free slot of the cache (the paper's
+ * future work, Sec. 5), (iii) per-sequence shapes, one call per shape.  mask_mode must be
+ * PEVLM_MASK_PEVLM; first_key_row >= S and first_key_row + N*B <= cache_rows, else PEVLM_EINVAL.
+ * batch strides: N*B rows for q / o / lse, cache_rows rows for the caches.  Workspace as for
+ * pevlm_parallel_prefill_attn.
+ */
+int pevlm_block_attn(const pevlm_shape_t* shape, const void* q_blocks, const void* k_cache,
+                     const void* v_cache, int64_t first_key_row, int64_t cache_rows, void* o, float* lse,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * KV-cache assembly [Eq. 5's key set s + c_all + q]: k_cache, v_cache [L, Hkv, d] receive
  * the video rows [0, S+N*B) from k_video / v_video and the question rows from k_question /
  * v_question [Q, Hkv, d].  K inputs are roped.  A source pointer may be NULL to skip that

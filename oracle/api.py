@@ -14,15 +14,24 @@ _lib = None
 
 class Shape(C.Structure):
     _fields_ = [("S", C.c_int64), ("B", C.c_int64), ("N", C.c_int64), ("Q", C.c_int64),
-                ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32), ("full_causal", C.c_int32)]
+                ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32), ("full_causal", C.c_int32),
+                ("B_last", C.c_int64)]
+
+    @property
+    def n_video(self):
+        if self.N <= 0:
+            return self.S
+        return self.S + (self.N - 1) * self.B + (self.B_last if self.B_last > 0 else self.B)
 
     @property
     def L(self):
-        return self.S + self.N * self.B + self.Q
+        return self.n_video + self.Q
 
 
-def make_shape(S, B, N, Q, Hq, Hkv, d, full_causal=False) -> Shape:
-    return Shape(S, B, N, Q, Hq, Hkv, d, 1 if full_causal else 0)
+def make_shape(S, B, N, Q, Hq, Hkv, d, full_causal=False, B_last=0) -> Shape:
+    """B_last: length of the last context block when the video does not divide evenly (0 = B)."""
+    assert 0 <= B_last <= B
+    return Shape(S, B, N, Q, Hq, Hkv, d, 1 if full_causal else 0, B_last)
 
 
 def lib():

@@ -11,19 +11,21 @@ from __future__ import annotations
 import numpy as np
 
 
-def segment_ids(S, B, N, Q):
-    """-1 for sink tokens, block index for context tokens, N for question tokens."""
-    seg = np.empty(S + N * B + Q, dtype=np.int64)
-    seg[:S] = -1
-    for b in range(N):
-        seg[S + b * B:S + (b + 1) * B] = b
-    seg[S + N * B:] = N
+def segment_ids(S, B, N, Q, B_last=0):
+    """-1 for sink tokens, block index for context tokens, N for question tokens.  The last
+    context block may be shorter than the others (B_last tokens; 0 = B)."""
+    lens = [B] * N
+    if N > 0 and B_last > 0:
+        lens[-1] = B_last
+    seg = np.concatenate([np.full(S, -1, dtype=np.int64)] +
+                         [np.full(n, b, dtype=np.int64) for b, n in enumerate(lens)] +
+                         [np.full(Q, N, dtype=np.int64)])
     return seg
 
 
-def dense_mask(S, B, N, Q, full_causal=False):
-    L = S + N * B + Q
-    seg = segment_ids(S, B, N, Q)
+def dense_mask(S, B, N, Q, full_causal=False, B_last=0):
+    seg = segment_ids(S, B, N, Q, B_last)
+    L = len(seg)
     row = np.arange(L)[:, None]
     col = np.arange(L)[None, :]
     causal = col <= row

@@ -49,7 +49,16 @@ typedef struct {
     int64_t S, B, N, Q;   /* sink, block length, number of blocks, question length */
     int32_t Hq, Hkv, d;
     int32_t full_causal;  /* 0: PEVLM mask (Eq. 3-5); 1: plain causal attention (Eq. 1-2) */
+    int64_t B_last;       /* length of the last context block, 1 <= B_last <= B; 0 means B.  Sec. 3.2.1
+                             partitions the video uniformly and does not say what happens to a remainder:
+                             here the remainder forms one shorter last block */
 } oracle_shape_t;
+
+/* number of video tokens: sink + all context blocks */
+static int64_t video_len(const oracle_shape_t* sh) {
+    if (sh->N <= 0) return sh->S;
+    return sh->S + (sh->N - 1) * sh->B + (sh->B_last > 0 ? sh->B_last : sh->B);
+}
 
 static double bf16_to_f64(uint16_t b) {
     uint32_t u = (uint32_t)b << 16;
@@ -81,7 +90,7 @@ int oracle_num_threads(void) {
  * range r is [lo[r], hi[r]) in global token indices.
  */
 int oracle_visible(const oracle_shape_t* sh, int64_t t, int64_t lo[2], int64_t hi[2]) {
-    int64_t nv = sh->S + sh->N * sh->B;
+    int64_t nv = video_len(sh);
     if (sh->full_causal || t < sh->S || t >= nv) {
         /* sink rows (Eq. 3) and question rows (Eq. 5): every key up to and including t */
         lo[0] = 0; hi[0] = t + 1;
@@ -174,7 +183,7 @@ void oracle_attn_rows(const oracle_shape_t* sh, const uint16_t* q, const uint16_
     const int32_t d = sh->d, Hq = sh->Hq, Hkv = sh->Hkv;
     const int32_t G = Hq / Hkv;
     if (scale <= 0.0) scale = 1.0 / sqrt((double)d);
-    const int64_t L = sh->S + sh->N * sh->B + sh->Q;
+    const int64_t L = video_len(sh) + sh->Q;
     int64_t work = n_rows * Hq;
 #pragma omp parallel
     {
@@ -238,7 +247,7 @@ void oracle_weights_row(const oracle_shape_t* sh, const uint16_t* q, const uint1
     const int32_t d = sh->d, Hq = sh->Hq, Hkv = sh->Hkv;
     const int32_t g = h / (Hq / Hkv);
     if (scale <= 0.0) scale = 1.0 / sqrt((double)d);
-    const int64_t L = sh->S + sh->N * sh->B + sh->Q;
+    const int64_t L = video_len(sh) + sh->Q;
     for (int64_t j = 0; j < L; ++j) w[j] = 0.0;
     int64_t lo[2], hi[2];
     int nr = oracle_visible(sh, t, lo, hi);
@@ -294,7 +303,7 @@ void oracle_merge_lse(const double* o_parts, const double* lse_parts, int64_t n_
  */
 void oracle_assemble_kv(const oracle_shape_t* sh, const uint16_t* video, const uint16_t* question,
                         uint16_t* cache) {
-    int64_t nv = sh->S + sh->N * sh->B;
+    int64_t nv = video_len(sh);
     size_t row = (size_t)sh->Hkv * sh->d;
     for (int64_t t = 0; t < nv + sh->Q; ++t) {
         const uint16_t* src = (t < nv) ? video + (size_t)t * row : question + (size_t)(t - nv) * row;
@@ -308,11 +317,12 @@ void oracle_assemble_kv(const oracle_shape_t* sh, const uint16_t* video, const u
  * count that the paper's operation model uses (Eq. 6-10).
  */
 int64_t oracle_count_rect_pairs(const oracle_shape_t* sh) {
-    int64_t nv = sh->S + sh->N * sh->B, L = nv + sh->Q, total = 0;
+    int64_t nv = video_len(sh), L = nv + sh->Q, total = 0;
     for (int64_t t = 0; t < L; ++t) {
         int64_t lo[2], hi[2];
         int nr = oracle_visible(sh, t, lo, hi);
         int64_t seg_end = (t < sh->S) ? sh->S : (t < nv) ? sh->S + ((t - sh->S) / sh->B + 1) * sh->B : L;
+        if (t < nv && seg_end > nv) seg_end = nv;  /* shorter last block */
         hi[nr - 1] = seg_end;
         for (int r = 0; r < nr; ++r) total += hi[r] - lo[r];
     }
@@ -321,7 +331,7 @@ int64_t oracle_count_rect_pairs(const oracle_shape_t* sh) {
 
 /* Count of visible (row, key) pairs per head, by enumeration of the mask. */
 int64_t oracle_count_pairs(const oracle_shape_t* sh) {
-    int64_t L = sh->S + sh->N * sh->B + sh->Q, total = 0;
+    int64_t L = video_len(sh) + sh->Q, total = 0;
     for (int64_t t = 0; t < L; ++t) {
         int64_t lo[2], hi[2];
         int nr = oracle_visible(sh, t, lo, hi);

@@ -21,7 +21,7 @@ WS_PREFILL, WS_QUERY = 0, 1
 
 NOALLOC_SCRATCH_BYTES = 32 << 20
 
-EXPORTS = ["pevlm_rope_qk", "pevlm_rope_qk_mrope", "pevlm_parallel_prefill_attn", "pevlm_assemble_kv", "pevlm_query_attn",
+EXPORTS = ["pevlm_rope_qk", "pevlm_rope_qk_mrope", "pevlm_parallel_prefill_attn", "pevlm_block_attn", "pevlm_assemble_kv", "pevlm_query_attn",
            "pevlm_query_attn_noalloc",
            "pevlm_workspace_bytes", "pevlm_read_status", "pevlm_tile_stats", "pevlm_strerror",
            "pevlm_last_cuda_error"]
@@ -70,6 +70,8 @@ def lib():
         l.pevlm_rope_qk_mrope.argtypes = [sp, vp, vp, vp, vp, C.c_int64, vp, C.POINTER(C.c_int32), vp]
         l.pevlm_rope_qk_mrope.restype = C.c_int
         l.pevlm_parallel_prefill_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        l.pevlm_block_attn.argtypes = [sp, vp, vp, vp, C.c_int64, C.c_int64, vp, vp, vp, C.c_size_t, vp]
+        l.pevlm_block_attn.restype = C.c_int
         l.pevlm_assemble_kv.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp]
         l.pevlm_query_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         l.pevlm_query_attn_noalloc.argtypes = [sp, vp, vp, vp, vp, vp, vp]
@@ -121,6 +123,12 @@ def pevlm_parallel_prefill_attn(shape: Shape, q, k, v, o, lse, workspace):
     _check(lib().pevlm_parallel_prefill_attn(C.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                              _ptr(workspace), workspace.numel() * workspace.element_size(),
                                              _stream()), "pevlm_parallel_prefill_attn")
+
+
+def pevlm_block_attn(shape: Shape, q_blocks, k_cache, v_cache, first_key_row: int, cache_rows: int, o, lse, workspace):
+    _check(lib().pevlm_block_attn(C.byref(shape), _ptr(q_blocks), _ptr(k_cache), _ptr(v_cache), first_key_row,
+                                  cache_rows, _ptr(o), _ptr(lse), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream()), "pevlm_block_attn")
 
 
 def pevlm_assemble_kv(shape: Shape, k_video, v_video, k_question, v_question, k_cache, v_cache):

@@ -265,8 +265,12 @@ int pevlm_assemble_kv(const pevlm_shape_t* s, const void* k_video, const void* v
     return PEVLM_OK;
 }
 
-int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const void* k, const void* v, void* o, float* lse,
-                                void* workspace, size_t workspace_bytes, void* stream) {
+// Prefill attention launches.  blocks_only = false: the whole video stream [sink | N blocks] (or full causal).
+// blocks_only = true: N blocks whose K/V sit at rows [first_key_row, first_key_row + N*B) of a cache of cache_rows
+// rows whose first S rows are the sink; q / o / lse cover the N*B block rows only and the sink rows are not computed.
+static int prefill_common(const pevlm_shape_t* s, const void* q, const void* k, const void* v, void* o, float* lse,
+                          void* workspace, size_t workspace_bytes, void* stream, bool blocks_only,
+                          int64_t first_key_row, int64_t cache_rows) {
     int rc = check_shape(s);
     if (rc != PEVLM_OK) return rc;
     if (!q || !k || !v || !o) return PEVLM_EINVAL;
@@ -274,7 +278,15 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
     if (!workspace || workspace_bytes < pevlm_workspace_bytes(s, PEVLM_WS_PREFILL)) return PEVLM_EWORKSPACE;
     if (!aligned256(workspace)) return PEVLM_EALIGN;
     const int64_t nv = n_video(s);
-    if (nv == 0) return PEVLM_OK;
+    const int64_t block_rows = static_cast<int64_t>(s->num_blocks) * s->block_len;
+    if (blocks_only) {
+        if (s->mask_mode != PEVLM_MASK_PEVLM) return PEVLM_EINVAL;
+        if (first_key_row < s->sink_len || first_key_row + block_rows > cache_rows || cache_rows > (1ll << 30))
+            return PEVLM_EINVAL;
+        if (block_rows == 0) return PEVLM_OK;
+    } else if (nv == 0) {
+        return PEVLM_OK;
+    }
     rc = check_device();
     if (rc != PEVLM_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -282,6 +294,8 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
     if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
 
     const int d = s->head_dim;
+    const int64_t q_rows = blocks_only ? block_rows : nv;   // rows of q, o, lse
+    const int64_t kv_rows = blocks_only ? cache_rows : nv;  // rows of k, v
     AttnParams p;
     memset(&p, 0, sizeof(p));
     p.mode = 0;
@@ -291,12 +305,15 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
         p.S = s->sink_len; p.B = s->num_blocks > 0 ? s->block_len : 0; p.N = s->num_blocks;
     }
     p.n_video = static_cast<int>(nv);
+    p.blk_key0 = blocks_only ? static_cast<int>(first_key_row) : p.S;
+    p.blk_q0 = blocks_only ? 0 : p.S;
+    p.q_rows = static_cast<int>(q_rows);
     p.Q = s->query_len;
     p.L = static_cast<int>(nv + s->query_len);
     p.Hq = s->num_q_heads; p.Hkv = s->num_kv_heads; p.G = p.Hq / p.Hkv;
     p.tiles_sink = (p.S + kTile - 1) / kTile;
     p.tiles_block = p.N > 0 ? (p.B + kTile - 1) / kTile : 0;
-    const SegPlan pb = plan_segment(p.N > 0 ? p.B : 0, p.G), ps = plan_segment(p.S, p.G);
+    const SegPlan pb = plan_segment(p.N > 0 ? p.B : 0, p.G), ps = plan_segment(blocks_only ? 0 : p.S, p.G);
     p.pairs_block = pb.pairs;
     p.pairs_sink = ps.pairs;
     p.tail_rows_block = pb.tail_rows; p.tail_heads_block = pb.tail_heads; p.tail_tiles_block = pb.tail_tiles;
@@ -307,18 +324,18 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
     p.scale_log2 = p.scale * 1.4426950408889634f;
     p.hdr = static_cast<WorkspaceHeader*>(workspace);
     for (int b = 0; b < s->batch; ++b) {
-        const int64_t qoff = static_cast<int64_t>(b) * nv * p.Hq * d, koff = static_cast<int64_t>(b) * nv * p.Hkv * d;
+        const int64_t qoff = static_cast<int64_t>(b) * q_rows * p.Hq * d, koff = static_cast<int64_t>(b) * kv_rows * p.Hkv * d;
         CUtensorMap tq, tq_tb, tq_ts, tk, tv;
         const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q) + qoff;
-        if ((rc = make_tmap(&tq, qb, nv, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tq, qb, q_rows, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
         tq_tb = tq;
         tq_ts = tq;
-        if (pb.tail_tiles > 0 && (rc = make_tmap(&tq_tb, qb, nv, p.Hq, d, pb.tail_heads, pb.tail_rows)) != PEVLM_OK) return rc;
-        if (ps.tail_tiles > 0 && (rc = make_tmap(&tq_ts, qb, nv, p.Hq, d, ps.tail_heads, ps.tail_rows)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, nv, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if (pb.tail_tiles > 0 && (rc = make_tmap(&tq_tb, qb, q_rows, p.Hq, d, pb.tail_heads, pb.tail_rows)) != PEVLM_OK) return rc;
+        if (ps.tail_tiles > 0 && (rc = make_tmap(&tq_ts, qb, q_rows, p.Hq, d, ps.tail_heads, ps.tail_rows)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k) + koff, kv_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, kv_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         p.o = static_cast<__nv_bfloat16*>(o) + qoff;
-        p.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * nv : nullptr;
+        p.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * q_rows : nullptr;
         if (b > 0) {  // every launch starts its work counter at zero; the status word is kept
             e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
             if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
@@ -327,6 +344,18 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const voi
         if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
     }
     return PEVLM_OK;
+}
+
+int pevlm_parallel_prefill_attn(const pevlm_shape_t* s, const void* q, const void* k, const void* v, void* o, float* lse,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    return prefill_common(s, q, k, v, o, lse, workspace, workspace_bytes, stream, false, 0, 0);
+}
+
+int pevlm_block_attn(const pevlm_shape_t* s, const void* q_blocks, const void* k_cache, const void* v_cache,
+                     int64_t first_key_row, int64_t cache_rows, void* o, float* lse, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    return prefill_common(s, q_blocks, k_cache, v_cache, o, lse, workspace, workspace_bytes, stream, true,
+                          first_key_row, cache_rows);
 }
 
 int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void* k_cache, const void* v_cache, void* o,

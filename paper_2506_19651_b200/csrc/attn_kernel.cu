@@ -82,13 +82,14 @@ __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
 __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem& it) {
     it.split = 0;
     if (p.mode == 0) {
-        int seg_start, seg_len, tiles, pi, g, tail_rows, tail_heads, tail_tiles, qmap_tail;
+        int seg_start, seg_q0, seg_len, tiles, pi, g, tail_rows, tail_heads, tail_tiles, qmap_tail;
         if (w < p.items_block) {
             const int combo = w / p.pairs_block;
             pi = w % p.pairs_block;
             const int blk = combo / p.Hkv;
             g = combo % p.Hkv;
-            seg_start = p.S + blk * p.B;
+            seg_start = p.blk_key0 + blk * p.B;  // key rows of the block
+            seg_q0 = p.blk_q0 + blk * p.B;       // its rows in q / o
             seg_len = p.B;
             tiles = p.tiles_block;
             tail_rows = p.tail_rows_block; tail_heads = p.tail_heads_block; tail_tiles = p.tail_tiles_block;
@@ -99,6 +100,7 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             g = w2 / p.pairs_sink;
             pi = w2 % p.pairs_sink;
             seg_start = 0;
+            seg_q0 = 0;
             seg_len = p.S;
             tiles = p.tiles_sink;
             tail_rows = p.tail_rows_sink; tail_heads = p.tail_heads_sink; tail_tiles = p.tail_tiles_sink;
@@ -136,9 +138,9 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
                 s.qmap = 0;
                 s.box_rows = kTile;
             }
-            s.q_tok0 = seg_start + qt * kTile;
-            s.limit0 = s.q_tok0;
-            s.b_end = min(s.q_tok0 + kTile, seg_start + seg_len);
+            s.q_tok0 = seg_q0 + qt * kTile;
+            s.limit0 = seg_start + qt * kTile;
+            s.b_end = min(s.limit0 + kTile, seg_start + seg_len);
             s.nt = s.valid ? it.na + cdiv(s.b_end - it.b_start, kTile) : 0;
         }
     } else {
@@ -631,7 +633,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 }
                 if (row_ok) {
                     if (p.mode == 0) {
-                        if (p.lse) p.lse[static_cast<size_t>(head) * p.n_video + tok] = lse_val;
+                        if (p.lse) p.lse[static_cast<size_t>(head) * p.q_rows + tok] = lse_val;
                     } else {
                         p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
                     }

@@ -27,6 +27,9 @@ struct AttnParams {
     int32_t mode;
     int32_t S, B, N;        // prefill geometry (full causal: S = 0, B = n_video, N = 1)
     int32_t n_video;        // S + N*B
+    int32_t blk_key0;       // mode 0: K/V row of the first context block (S, or the cache row of a block range)
+    int32_t blk_q0;         // mode 0: row of q / o where the first context block starts (S, or 0 for a block range)
+    int32_t q_rows;         // mode 0: rows of q / o = row stride of lse
     int32_t Q, L;           // question length, total length
     int32_t Hq, Hkv, G;
     int32_t tiles_sink;     // ceil(S / 128)

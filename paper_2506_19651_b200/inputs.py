@@ -36,14 +36,17 @@ class Workload:
     outliers: bool    # first 4 sink K rows x8
     seed: int
     layers: int = 1
+    B_last: int = 0   # length of the last context block when the video does not divide evenly (0 = B)
 
     @property
     def n_video(self) -> int:
-        return self.S + self.N * self.B
+        if self.N <= 0:
+            return self.S
+        return self.S + (self.N - 1) * self.B + (self.B_last or self.B)
 
     @property
     def L(self) -> int:
-        return self.S + self.N * self.B + self.Q
+        return self.n_video + self.Q
 
     def with_(self, **kw) -> "Workload":
         return replace(self, **kw)

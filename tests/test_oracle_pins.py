@@ -67,6 +67,48 @@ def test_oracle_vs_dense_mask(S, B, N, Q, Hq, Hkv, d):
     np.testing.assert_allclose(lse, lse_ref, rtol=0, atol=1e-11)
 
 
+# ---- shorter last context block (a video that does not divide evenly; Sec. 3.2.1 is silent) ----
+
+@pytest.mark.parametrize("S,B,N,Q,B_last,Hq,Hkv,d", [(3, 4, 3, 2, 1, 2, 1, 4), (8, 16, 3, 5, 7, 4, 2, 8),
+                                                     (0, 5, 2, 3, 4, 2, 2, 4), (6, 9, 1, 2, 5, 2, 1, 8)])
+def test_ragged_last_block_vs_dense_mask_and_counts(S, B, N, Q, B_last, Hq, Hkv, d):
+    w = inputs.Workload("t", S, B, N, Q, Hq, Hkv, d, 1e4, False, 13, B_last=B_last)
+    assert w.n_video == S + (N - 1) * B + B_last
+    q, k, v = inputs.make_qkv(w)
+    qr, kr = api.rope(q, 1e4), api.rope(k, 1e4)
+    sh = api.make_shape(S, B, N, Q, Hq, Hkv, d, B_last=B_last)
+    assert sh.L == w.L
+    o, lse = api.attn_rows(sh, qr, kr, v, all_rows(w.L))
+    mask = dense.dense_mask(S, B, N, Q, B_last=B_last)
+    assert mask.shape == (w.L, w.L)
+    o_ref, lse_ref, _ = dense.dense_attention(qr, kr, v, mask)
+    np.testing.assert_allclose(o, o_ref, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(lse, lse_ref, rtol=0, atol=1e-11)
+    # closed-form pair counts: the last block contributes B_last*S + tri(B_last) (Eq. 8 with its own length)
+    tri = lambda n: n * (n + 1) // 2
+    nv = w.n_video
+    want = tri(S) + (N - 1) * (B * S + tri(B)) + B_last * S + tri(B_last) + Q * nv + tri(Q)
+    assert api.count_pairs(sh) == want == int(mask.sum())
+    want_rect = S * S + (N - 1) * B * (S + B) + B_last * (S + B_last) + Q * w.L
+    assert api.count_rect_pairs(sh) == want_rect
+    # zero keys: LSE = ln(#visible) (row r of the last block sees S + r + 1 keys)
+    o0, lse0 = api.attn_rows(sh, q, np.zeros_like(k), v, all_rows(w.L))
+    first_last = S + (N - 1) * B
+    for t in range(first_last, nv):
+        assert abs(lse0[t, 0] - math.log(S + (t - first_last) + 1)) < 1e-12
+    for t in range(nv, w.L):
+        assert abs(lse0[t, 0] - math.log(t + 1)) < 1e-12
+
+
+def test_ragged_last_block_equal_to_uniform_when_lengths_agree():
+    S, B, N, Q, Hq, Hkv, d = 4, 6, 3, 2, 2, 1, 4
+    w, _, _, v, qr, kr = small_stream(S, B, N, Q, Hq, Hkv, d)
+    a = api.attn_rows(api.make_shape(S, B, N, Q, Hq, Hkv, d), qr, kr, v, all_rows(w.L))
+    b = api.attn_rows(api.make_shape(S, B, N, Q, Hq, Hkv, d, B_last=B), qr, kr, v, all_rows(w.L))
+    np.testing.assert_array_equal(a[0], b[0])
+    np.testing.assert_array_equal(a[1], b[1])
+
+
 # ---- P2: sink rows equal full-attention rows (Eq. 3) ---------------------------------
 
 def test_p2_sink_rows_equal_full_attention():
@@ -326,17 +368,18 @@ def test_p8_merge_all_empty_is_minus_inf():
 
 # ---- P9: literal triple loop on a tiny shape (Eq. 1, Eq. 3-5) ------------------------
 
-def _literal(S, B, N, Q, Hq, Hkv, d, q, k, v):
-    L = S + N * B + Q
+def _literal(S, B, N, Q, Hq, Hkv, d, q, k, v, B_last=0):
+    nv = S + (N - 1) * B + (B_last or B) if N > 0 else S
+    L = nv + Q
     G = Hq // Hkv
     o = [[[0.0] * d for _ in range(Hq)] for _ in range(L)]
     lse = [[0.0] * Hq for _ in range(L)]
     for t in range(L):
         if t < S:
             keys = [j for j in range(S) if j <= t]                          # Eq. 3
-        elif t < S + N * B:
+        elif t < nv:
             i = (t - S) // B
-            own = range(S + i * B, S + (i + 1) * B)
+            own = range(S + i * B, min(S + (i + 1) * B, nv))
             keys = list(range(S)) + [j for j in own if j <= t]              # Eq. 4
         else:
             keys = [j for j in range(L) if j <= t]                          # Eq. 5
@@ -350,12 +393,15 @@ def _literal(S, B, N, Q, Hq, Hkv, d, q, k, v):
     return np.array(o), np.array(lse)
 
 
-@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d", [(3, 4, 2, 2, 2, 1, 4), (2, 3, 3, 1, 4, 2, 2)])
-def test_p9_literal_loops(S, B, N, Q, Hq, Hkv, d):
-    w, _, _, v, qr, kr = small_stream(S, B, N, Q, Hq, Hkv, d)
-    o, lse = api.attn_rows(api.make_shape(S, B, N, Q, Hq, Hkv, d), qr, kr, v, all_rows(w.L))
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d,B_last", [(3, 4, 2, 2, 2, 1, 4, 0), (2, 3, 3, 1, 4, 2, 2, 0),
+                                                     (3, 4, 3, 2, 2, 1, 4, 2)])
+def test_p9_literal_loops(S, B, N, Q, Hq, Hkv, d, B_last):
+    w = inputs.Workload("t", S, B, N, Q, Hq, Hkv, d, 1e4, False, 11, B_last=B_last)
+    _, k, v = inputs.make_qkv(w)
+    qr, kr = api.rope(inputs.make_qkv(w)[0], 1e4), api.rope(k, 1e4)
+    o, lse = api.attn_rows(api.make_shape(S, B, N, Q, Hq, Hkv, d, B_last=B_last), qr, kr, v, all_rows(w.L))
     o_ref, lse_ref = _literal(S, B, N, Q, Hq, Hkv, d, dense.bits_to_f64(qr).tolist(),
-                              dense.bits_to_f64(kr).tolist(), dense.bits_to_f64(v).tolist())
+                              dense.bits_to_f64(kr).tolist(), dense.bits_to_f64(v).tolist(), B_last)
     np.testing.assert_allclose(o, o_ref, rtol=0, atol=1e-12)
     np.testing.assert_allclose(lse, lse_ref, rtol=0, atol=1e-12)
     # first row sees one key: O = V[0], LSE = its score

@@ -106,6 +106,15 @@ def test_argument_errors_before_launch(lib):
     assert lib.pevlm_rope_qk_mrope(C.byref(good), odd, None, odd, None, 8, p16, sec_ok, None) == pb.PEVLM_EALIGN
     assert lib.pevlm_assemble_kv(C.byref(good), p16, None, None, None, None, None, None) == pb.PEVLM_EINVAL
     assert lib.pevlm_query_attn(C.byref(good), p16, p16, p16, p16, None, ws, 16, None) == pb.PEVLM_EWORKSPACE
+    # block range: must start at or after the sink and end inside the cache; PEVLM mask only
+    g = lib.pevlm_block_attn
+    nb = good.num_blocks * good.block_len
+    assert g(C.byref(good), p16, p16, p16, 63, 64 + nb, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
+    assert g(C.byref(good), p16, p16, p16, 64, 64 + nb - 1, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
+    assert g(C.byref(good), p16, p16, odd, 64, 64 + nb, p16, None, ws, 1 << 20, None) == pb.PEVLM_EALIGN
+    assert g(C.byref(good), p16, p16, p16, 64, 64 + nb, p16, None, None, 0, None) == pb.PEVLM_EWORKSPACE
+    fc = pb.make_shape(64, 128, 4, 32, 4, 2, 64, mask_mode=pb.MASK_FULL_CAUSAL)
+    assert g(C.byref(fc), p16, p16, p16, 64, 64 + nb, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -378,29 +378,31 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             for (int x = 0; x < 2; ++x)
                 if (nt[x] > 0) wait(bar_q_full + 8 * x, q_uses[x] & 1, kWaitQ);
             tc_fence_after_sync();
-            // order on the tensor pipe: QK0(j) PV1(j-1) QK1(j) PV0(j): while one query tile is in its
-            // softmax the other one's MMAs run
-            for (int j = 0; j <= nt_max; ++j) {
-                if (j < nt_max) {
-                    wait_full(2 * j);
-                    tc_fence_after_sync();
-                    if (j < nt[0]) issue_qk(0, j);
+            // Order on the tensor pipe: QK0(0) QK1(0), then per key tile j: PV0(j) QK0(j+1) PV1(j) QK1(j+1).
+            // While one query tile is in its softmax the other one's MMAs run.  PV_x(j) and QK_x(j+1) go out
+            // back to back: everything they wait for except the probabilities (V(j), K(j+1)) is waited for
+            // before the wait on P_x(j), so the scores of the next tile follow the probabilities of this one
+            // through the pipe without a gap.
+            if (nt_max > 0) {
+                wait_full(0);
+                if (nt[0] > 0) issue_qk(0, 0);
+                if (nt[1] > 0) issue_qk(1, 0);
+                commit_empty(0);  // K(0) consumed
+            }
+            for (int j = 0; j < nt_max; ++j) {
+                const bool more = j + 1 < nt_max;
+                wait_full(2 * j + 1);             // V(j)
+                if (more) wait_full(2 * j + 2);   // K(j+1)
+                if (j < nt[0]) {
+                    issue_pv(0, j);
+                    if (j + 1 < nt[0]) issue_qk(0, j + 1);
                 }
-                if (j > 0) {
-                    if (j - 1 < nt[1]) {
-                        wait_full(2 * (j - 1) + 1);
-                        issue_pv(1, j - 1);
-                    }
-                    commit_empty(2 * (j - 1) + 1);  // V(j-1) consumed
+                if (j < nt[1]) {
+                    issue_pv(1, j);
+                    if (j + 1 < nt[1]) issue_qk(1, j + 1);
                 }
-                if (j < nt_max) {
-                    if (j < nt[1]) issue_qk(1, j);
-                    commit_empty(2 * j);  // K(j) consumed
-                    if (j < nt[0]) {
-                        wait_full(2 * j + 1);
-                        issue_pv(0, j);
-                    }
-                }
+                commit_empty(2 * j + 1);            // V(j) consumed
+                if (more) commit_empty(2 * j + 2);  // K(j+1) consumed
             }
             ring_base += 2 * nt_max;
 #pragma unroll

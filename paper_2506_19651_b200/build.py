@@ -37,6 +37,8 @@ def _stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     extra = ["-DPEVLM_PROFILE"] if os.environ.get("PEVLM_PROFILE") == "1" else []
+    if os.environ.get("PEVLM_TRACE") == "1":   # time stamps of the kernel's hand-offs, read by timeline.py
+        extra.append("-DPEVLM_TRACE")
     if not force and not _stale():
         return LIB
     objs = []

@@ -77,6 +77,25 @@ struct WorkItem {
     QSlot s[2];
 };
 
+// Optional time stamps (-DPEVLM_TRACE): clock64 at the hand-offs of CTA 0's first work item, key tiles
+// [kTraceJ0, kTraceJ0 + 16), read back through pevlm_debug_trace (see timeline.py).  Events: 0/1 scores of
+// tile 0/1 seen by the softmax, 2/3 probabilities handed over, 4 QK0 issue starts, 5 QK0 issued,
+// 6 probabilities of tile 0 seen by the MMA warp, 7 PV0 issued.
+#ifdef PEVLM_TRACE
+__device__ unsigned g_trace[8][16];
+constexpr int kTraceJ0 = 8;
+#define PEVLM_STAMP(ev, j, cond)                                                                \
+    do {                                                                                        \
+        if ((cond) && blockIdx.x == 0 && k == 0 && (j) >= kTraceJ0 && (j) < kTraceJ0 + 16)      \
+            g_trace[ev][(j) - kTraceJ0] = static_cast<unsigned>(clock64());                     \
+    } while (0)
+extern "C" int pevlm_debug_trace(unsigned* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
+}
+#else
+#define PEVLM_STAMP(ev, j, cond) do {} while (0)
+#endif
+
 __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
 
 __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem& it) {
@@ -340,10 +359,12 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             auto commit_empty = [&](int idx) { mma_commit_elect(bar_empty + 8 * ((ring_base + idx) % kRing)); };
             // S_x = Q_x K(j)^T
             auto issue_qk = [&](int x, int j) {
+                PEVLM_STAMP(4, j, lane == 0 && x == 0);
                 const int n_mma = (valid_of(x, j) + 15) & ~15;
                 const uint32_t idesc = make_idesc_bf16(kTile, n_mma, false);
                 mma_ss_batch<D / 16>(tmem_base + x * 128, desc_lo(smem_base + (x ? L::kQ1 : L::kQ0), 16),
                                      desc_lo(ring_addr(2 * j), 16), idesc);
+                PEVLM_STAMP(5, j, lane == 0 && x == 0);
                 mma_commit_elect(bar_s_full + 8 * x);
                 if (j == nt[x] - 1) mma_commit_elect(bar_q_free + 8 * x);  // last use of this Q tile
             };
@@ -356,6 +377,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
 #ifdef PEVLM_PROFILE
                 prof_po += static_cast<unsigned>(clock64()) - prof_a;
 #endif
+                PEVLM_STAMP(6, j, lane == 0 && x == 0);
                 // the previous item's output must have left TMEM before O is overwritten
                 if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWaitOFree);
                 tc_fence_after_sync();
@@ -371,6 +393,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                         mma_ts_elect(d_tmem, a_tmem + ks * 8, make_smem_desc_sw128(sv + ks * 2048, L::kPanelBytes, 1024), idesc,
                                      (j > 0) || (ks > 0));
                 }
+                PEVLM_STAMP(7, j, lane == 0 && x == 0);
                 // o_done: the item's accumulator is complete (one phase per item, for the epilogue)
                 if (j == nt[x] - 1) mma_commit_elect(bar_o_done + 8 * x);
             };
@@ -460,6 +483,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 prof_t1 = static_cast<unsigned>(clock64());
                 prof_wait += prof_t1 - prof_t2;
 #endif
+                PEVLM_STAMP(0 + x, j, (tid & 127) == 0);
                 tc_fence_after_sync();
                 // all 128 scores of the row in registers: one round trip to TMEM
                 uint32_t r[kTile];
@@ -542,6 +566,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(my_po);
+                PEVLM_STAMP(2 + x, j, (tid & 127) == 0);
 #ifdef PEVLM_PROFILE
                 prof_t2 = static_cast<unsigned>(clock64());
                 prof_busy += prof_t2 - prof_t1;

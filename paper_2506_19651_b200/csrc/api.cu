@@ -6,6 +6,7 @@
 #include <cstring>
 
 #include "internal.h"
+#include <cstdlib>
 
 namespace pevlm {
 
@@ -318,7 +319,15 @@ static int prefill_common(const pevlm_shape_t* s, const void* q, const void* k, 
     p.pairs_sink = ps.pairs;
     p.tail_rows_block = pb.tail_rows; p.tail_heads_block = pb.tail_heads; p.tail_tiles_block = pb.tail_tiles;
     p.tail_rows_sink = ps.tail_rows; p.tail_heads_sink = ps.tail_heads; p.tail_tiles_sink = ps.tail_tiles;
-    p.items_block = p.N * p.Hkv * p.pairs_block;
+#ifndef PEVLM_ORDER_CHUNKS
+#define PEVLM_ORDER_CHUNKS 1
+#endif
+    int want_chunks = PEVLM_ORDER_CHUNKS;
+    if (const char* e_chunks = getenv("PEVLM_EXP_CHUNKS")) want_chunks = atoi(e_chunks);  // EXPERIMENT
+    const int chunks = p.pairs_block > 0 ? (want_chunks < p.pairs_block ? want_chunks : p.pairs_block) : 1;
+    p.pair_chunk = p.pairs_block > 0 ? (p.pairs_block + chunks - 1) / chunks : 1;
+    const int n_chunks = p.pairs_block > 0 ? (p.pairs_block + p.pair_chunk - 1) / p.pair_chunk : 0;
+    p.items_block = p.N * p.Hkv * p.pair_chunk * n_chunks;
     p.n_items = p.items_block + p.Hkv * p.pairs_sink;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;

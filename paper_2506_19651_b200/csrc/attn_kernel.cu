@@ -103,8 +103,15 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
     if (p.mode == 0) {
         int seg_start, seg_q0, seg_len, tiles, pi, g, tail_rows, tail_heads, tail_tiles, qmap_tail;
         if (w < p.items_block) {
-            const int combo = w / p.pairs_block;
-            pi = w % p.pairs_block;
+            // Order of the items: the pair list of a (block, kv head), heaviest first, is cut into chunks of
+            // pair_chunk pairs; chunk-major, then (block, kv head), then the pairs of the chunk.  CTAs that run
+            // at the same time then share few K/V tiles' worth of L2 traffic, and the launch ends on the
+            // lightest chunk of every (block, kv head) rather than on the last block's whole list.  A pair
+            // index past the end of the list (padding of the last chunk) is an empty item.
+            const int per_chunk = p.N * p.Hkv * p.pair_chunk;
+            const int r = w % per_chunk;
+            const int combo = r / p.pair_chunk;
+            pi = (w / per_chunk) * p.pair_chunk + r % p.pair_chunk;
             const int blk = combo / p.Hkv;
             g = combo % p.Hkv;
             seg_start = p.blk_key0 + blk * p.B;  // key rows of the block
@@ -211,6 +218,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int s_item[2];
+    __shared__ WorkItem s_decoded[2];  // the producer decodes an item once; every role copies it from here
     __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a short
     __shared__ float s_final_m[2][2][kTile];  // item while the previous item's epilogue is still running
 
@@ -265,9 +273,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
     };
     // consumer side of the item queue: k-th item of this CTA, -1 = no more work
-    auto next_item = [&](int k) {
+    auto next_item = [&](int k, WorkItem& it) {
         wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
         const int w = s_item[k & 1];
+        if (w >= 0) it = s_decoded[k & 1];
         mbar_arrive(bar_item_free + 8 * (k & 1));
         return w;
     };
@@ -286,10 +295,13 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 if (w >= p.n_items || abort_flag != 0 || *reinterpret_cast<volatile int32_t*>(&p.hdr->status) != 0) w = -1;
                 if (k >= 2) wait(bar_item_free + 8 * (k & 1), ((k >> 1) - 1) & 1, kWaitItemFree);
                 s_item[k & 1] = w;
-                mbar_arrive(bar_item_full + 8 * (k & 1));
-                if (w < 0) break;
                 WorkItem it;
-                decode_item(p, w, it);
+                if (w >= 0) {
+                    decode_item(p, w, it);
+                    s_decoded[k & 1] = it;
+                }
+                mbar_arrive(bar_item_full + 8 * (k & 1));  // release: the item and its decoded form are visible
+                if (w < 0) break;
                 const int nt_max = max(it.s[0].nt, it.s[1].nt);
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
@@ -331,11 +343,11 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             // every lane reads the item, one lane releases the queue slot
             wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
             const int w = s_item[k & 1];
+            WorkItem it;
+            if (w >= 0) it = s_decoded[k & 1];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_item_free + 8 * (k & 1));
             if (w < 0) break;
-            WorkItem it;
-            decode_item(p, w, it);
             const int nt[2] = {it.s[0].nt, it.s[1].nt};
             const int nt_max = max(nt[0], nt[1]);
             // keys in the last tile of the shared range and of each slot's own range (every other
@@ -459,10 +471,9 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         unsigned prof_ld = 0, prof_exp = 0;
 #endif
         for (int k = 0;; ++k) {
-            const int w = next_item(k);
-            if (w < 0) break;
             WorkItem it;
-            decode_item(p, w, it);
+            const int w = next_item(k, it);
+            if (w < 0) break;
             // this slot's scalars, in registers
             const int nt = x ? it.s[1].nt : it.s[0].nt;
             const int item_ring_base = ring_base;
@@ -599,10 +610,9 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_done / o_free)
         for (int k = 0;; ++k) {
-            const int w = next_item(k);
-            if (w < 0) break;
             WorkItem it;
-            decode_item(p, w, it);
+            const int w = next_item(k, it);
+            if (w < 0) break;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 const QSlot& s = it.s[x];

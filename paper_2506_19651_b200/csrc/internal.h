@@ -36,7 +36,8 @@ struct AttnParams {
     int32_t tiles_block;    // ceil(B / 128)
     int32_t pairs_block;    // ceil(G * tiles_block / 2) query-tile pairs per (block, kv head)
     int32_t pairs_sink;     // ceil(G * tiles_sink / 2) query-tile pairs per kv head
-    int32_t items_block;    // N * Hkv * pairs_block work items over the context blocks
+    int32_t pair_chunk;     // pairs of one (block, kv head) handed out together (see decode_item)
+    int32_t items_block;    // work items over the context blocks, padded: N * Hkv * pair_chunk * chunks
     int32_t n_items;        // all work items of the launch
     // ragged last query tile of a segment (len % 128 rows): the tails of tail_heads q heads of one kv
     // group are packed into one 128-row tile, tail_tiles such tiles per (segment, kv head); 0 = no packing

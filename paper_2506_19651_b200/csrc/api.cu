@@ -6,7 +6,6 @@
 #include <cstring>
 
 #include "internal.h"
-#include <cstdlib>
 
 namespace pevlm {
 
@@ -319,13 +318,14 @@ static int prefill_common(const pevlm_shape_t* s, const void* q, const void* k, 
     p.pairs_sink = ps.pairs;
     p.tail_rows_block = pb.tail_rows; p.tail_heads_block = pb.tail_heads; p.tail_tiles_block = pb.tail_tiles;
     p.tail_rows_sink = ps.tail_rows; p.tail_heads_sink = ps.tail_heads; p.tail_tiles_sink = ps.tail_tiles;
-#ifndef PEVLM_ORDER_CHUNKS
-#define PEVLM_ORDER_CHUNKS 1
-#endif
-    int want_chunks = PEVLM_ORDER_CHUNKS;
-    if (const char* e_chunks = getenv("PEVLM_EXP_CHUNKS")) want_chunks = atoi(e_chunks);  // EXPERIMENT
-    const int chunks = p.pairs_block > 0 ? (want_chunks < p.pairs_block ? want_chunks : p.pairs_block) : 1;
-    p.pair_chunk = p.pairs_block > 0 ? (p.pairs_block + chunks - 1) / chunks : 1;
+    // How many pairs of one (block, kv head) are handed out together (decode_item): the whole list keeps the CTAs
+    // that run at the same time on few K/V tiles (best for long blocks); short blocks (at most 4 query tiles)
+    // run faster when pairs of equal length are handed out together across all blocks, and a launch with few
+    // items per SM balances best with single pairs, heaviest first.  Thresholds from measurements on B200.
+    int want_pc = p.pairs_block;
+    if (p.tiles_block <= 4) want_pc = p.G / 2 > 0 ? p.G / 2 : 1;
+    else if (static_cast<int64_t>(p.N) * p.Hkv * p.pairs_block < 16 * kNumSms) want_pc = 1;
+    p.pair_chunk = p.pairs_block > 0 ? (want_pc < p.pairs_block ? want_pc : p.pairs_block) : 1;
     const int n_chunks = p.pairs_block > 0 ? (p.pairs_block + p.pair_chunk - 1) / p.pair_chunk : 0;
     p.items_block = p.N * p.Hkv * p.pair_chunk * n_chunks;
     p.n_items = p.items_block + p.Hkv * p.pairs_sink;

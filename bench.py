@@ -420,7 +420,9 @@ def run_sweep(args):
     for F in (1, 2, 4, 8, 16, 32):
         w = inputs.sweep_workload(F)
         q, k, v = device_inputs(w)
+        sampler = ClockSampler(0)
         shape, per = time_layer(w, args.steps, args.warmup, q, k, v)
+        clocks = sampler.stop()
         pre = pb.pevlm_tile_stats(shape, pb.WS_PREFILL)
         t = per["prefill_attn"]
         useful = 4.0 * w.d * w.Hq * (visible_pairs(w) - (w.Q * w.n_video + w.Q * (w.Q + 1) // 2))
@@ -430,7 +432,9 @@ def run_sweep(args):
                           "active_tile_tflops": pre.flops / (t * 1e-3) / 1e12, "useful_tflops": useful / (t * 1e-3) / 1e12,
                           "frac_of_bf16_peak": pre.flops / (t * 1e-3) / 1e12 / peaks["bf16_tflops"],
                           "full_causal_active_gflop": pb.pevlm_tile_stats(fshape, pb.WS_PREFILL).flops / 1e9,
-                          "data": "synthetic (device-generated)"}))
+                          "clocks": clocks, "data": "synthetic (device-generated)"}))
+        del q, k, v
+        torch.cuda.empty_cache()
 
 
 def run_stack(args):

@@ -437,6 +437,54 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_sink_sweep(args):
+    """Sink-size sweep at fixed context blocks (the structure of the paper's sink-size study, Sec. 4.4): 15
+    blocks of 2,048 tokens, Qwen-shaped heads, sink of 0 .. 4,096 tokens.  One JSON line per sink size; the
+    last line times the multimodal RoPE against the plain one on the largest stream."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    for S in (0, 128, 256, 512, 1024, 2048, 4096):
+        w = inputs.Workload(f"sink_{S}", S, 2048, 15, 64, 28, 4, 128, 1e6, S > 0, inputs.WORKLOADS["c3_long"].seed + S)
+        q, k, v = device_inputs(w)
+        sampler = ClockSampler(0)
+        shape, per = time_layer(w, args.steps, args.warmup, q, k, v)
+        clocks = sampler.stop()
+        pre = pb.pevlm_tile_stats(shape, pb.WS_PREFILL)
+        t = per["prefill_attn"]
+        useful = 4.0 * w.d * w.Hq * (visible_pairs(w) - (w.Q * w.n_video + w.Q * (w.Q + 1) // 2))
+        print(json.dumps({"kind": "sink_sweep", "sink_len": S, "block_len": w.B, "num_blocks": w.N, "tokens": w.L,
+                          "ms_per_layer": sum(per.values()), "kernels_ms": per, "prefill_ms": t,
+                          "active_tile_tflops": pre.flops / (t * 1e-3) / 1e12, "useful_tflops": useful / (t * 1e-3) / 1e12,
+                          "frac_of_bf16_peak": pre.flops / (t * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                          "clocks": clocks, "data": "synthetic (device-generated)"}))
+        if S < 4096:
+            del q, k, v
+            torch.cuda.empty_cache()
+    # multimodal RoPE on the same stream: ids of a 16 x 16 token grid per frame after a 64-token text prefix
+    n = w.n_video
+    idx = torch.arange(n, device="cuda", dtype=torch.int32)
+    frame, inside = torch.div(idx, 256, rounding_mode="floor"), idx % 256
+    pos3 = torch.stack([64 + frame, 64 + torch.div(inside, 16, rounding_mode="floor"), 64 + inside % 16]).contiguous()
+    qo, ko = torch.empty_like(q[:n]), torch.empty_like(k[:n])
+    times = {}
+    for name, call in (("rope_plain", lambda: pb.pevlm_rope_qk(shape, q[:n], k[:n], qo, ko, 0, n)),
+                       ("rope_multimodal", lambda: pb.pevlm_rope_qk_mrope(shape, q[:n], k[:n], qo, ko, n, pos3, (16, 24, 24)))):
+        for _ in range(3):
+            call()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            call()
+        b.record()
+        torch.cuda.synchronize()
+        times[name] = a.elapsed_time(b) / args.steps
+    nbytes = 2.0 * n * (w.Hq + w.Hkv) * w.d * 2
+    print(json.dumps({"kind": "rope_forms", "tokens": n, "ms": times,
+                      "gbs": {k2: nbytes / (v2 * 1e-3) / 1e9 for k2, v2 in times.items()}}))
+
+
 def run_stack(args):
     """Attention of a whole prefill stack: every layer has its own seeded Q/K/V and its own KV cache."""
     import torch
@@ -482,6 +530,7 @@ def main():
     ap.add_argument("--skip-full-causal", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="block-size sweep: one JSON line per block size")
     ap.add_argument("--stack", action="store_true", help="28-layer attention stack: one JSON line")
+    ap.add_argument("--sink-sweep", action="store_true", help="sink-size sweep at fixed blocks, then the two RoPE forms")
     ap.add_argument("--layers", type=int, default=0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -490,6 +539,8 @@ def main():
         return run_sweep(args)
     if args.stack:
         return run_stack(args)
+    if args.sink_sweep:
+        return run_sink_sweep(args)
     if args.impl == "reference":
         run_reference(args, w)
     else:

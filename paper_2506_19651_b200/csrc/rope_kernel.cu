@@ -28,8 +28,10 @@ __device__ __forceinline__ uint32_t f64x2_to_bf16x2_bits(double lo, double hi) {
 // no block-level synchronisation; CTAs stride over groups of 256 / (d/16) token slots.  For short
 // token ranges (the question block) the heads of a token are split over `head_split` such thread
 // groups, each evaluating the token's angles itself, so the launch still fills the machine.
-// MROPE = true: the multimodal form, where a rotary pair's section picks the position component.
-template <int D, bool MROPE>
+// MODE 0: one position per token.  MODE 1, 2: the multimodal form, where a rotary pair's section picks the
+// position component; 1 when the section boundaries are multiples of 8 pairs (16/24/24 at d = 128), so that a
+// thread's 8 pairs share one component, 2 in general (a component per pair, more registers).
+template <int D, int MODE>
 __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constant__ RopeParams p) {
     constexpr int HALF = D / 2;
     constexpr int TPT = HALF / 8;                  // threads per token
@@ -44,12 +46,16 @@ __global__ void __launch_bounds__(kRopeThreads) rope_kernel(const __grid_constan
         const int64_t tok = slot / p.head_split;
         const int h_first = static_cast<int>(slot % p.head_split);
         int64_t pos = 0;
-        if (!MROPE) pos = p.pos_ids ? static_cast<int64_t>(p.pos_ids[tok]) : p.first_token + tok;
+        if (MODE == 0) pos = p.pos_ids ? static_cast<int64_t>(p.pos_ids[tok]) : p.first_token + tok;
+        if (MODE == 1) {
+            const int comp = i0 < p.sec_end0 ? 0 : i0 < p.sec_end1 ? 1 : 2;
+            pos = static_cast<int64_t>(p.pos3[comp * p.n_tokens + tok]);
+        }
         double cs[8], sn[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             int64_t pe = pos;
-            if (MROPE) {  // multimodal: the pair's section picks the temporal, height or width position
+            if (MODE == 2) {  // multimodal: the pair's section picks the temporal, height or width position
                 const int i = i0 + e;
                 const int comp = i < p.sec_end0 ? 0 : i < p.sec_end1 ? 1 : 2;
                 pe = static_cast<int64_t>(p.pos3[comp * p.n_tokens + tok]);
@@ -106,12 +112,15 @@ cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream) 
     const int64_t groups = (p.n_tokens * q.head_split + tok_per_cta - 1) / tok_per_cta;
     const int64_t cap = 148 * 8;  // whole waves of the 148 SMs; CTAs stride over the remaining groups
     const unsigned grid = static_cast<unsigned>(groups < cap ? groups : cap);
+    const int mode = !q.pos3 ? 0 : ((q.sec_end0 | q.sec_end1) & 7) == 0 ? 1 : 2;
     if (head_dim == 128) {
-        if (q.pos3) rope_kernel<128, true><<<grid, kRopeThreads, 0, stream>>>(q);
-        else rope_kernel<128, false><<<grid, kRopeThreads, 0, stream>>>(q);
+        if (mode == 0) rope_kernel<128, 0><<<grid, kRopeThreads, 0, stream>>>(q);
+        else if (mode == 1) rope_kernel<128, 1><<<grid, kRopeThreads, 0, stream>>>(q);
+        else rope_kernel<128, 2><<<grid, kRopeThreads, 0, stream>>>(q);
     } else {
-        if (q.pos3) rope_kernel<64, true><<<grid, kRopeThreads, 0, stream>>>(q);
-        else rope_kernel<64, false><<<grid, kRopeThreads, 0, stream>>>(q);
+        if (mode == 0) rope_kernel<64, 0><<<grid, kRopeThreads, 0, stream>>>(q);
+        else if (mode == 1) rope_kernel<64, 1><<<grid, kRopeThreads, 0, stream>>>(q);
+        else rope_kernel<64, 2><<<grid, kRopeThreads, 0, stream>>>(q);
     }
     return cudaGetLastError();
 }

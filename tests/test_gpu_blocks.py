@@ -23,6 +23,7 @@ def _status_ok(*workspaces):
     (0, 256, 2, 8, 255, 4, 4, 128),        # no sink
     (130, 260, 1, 5, 7, 14, 2, 128),       # the only block is the short one, G = 7 (packed tails)
     (784, 784, 5, 64, 392, 28, 4, 128),    # Qwen-shaped, half a block left over
+    (1568, 1568, 31, 128, 980, 28, 4, 128),  # the 50K-token shape with 5 of the last block's 8 frames (sampled rows)
 ])
 def test_ragged_last_block(S, B, N, Q, B_last, Hq, Hkv, d):
     import torch

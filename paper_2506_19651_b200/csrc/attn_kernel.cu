@@ -14,8 +14,9 @@
 //               O += P V (P from TMEM, V from shared memory), ping-ponging between the two
 //               query tiles so one is in the tensor cores while the other is in its softmax
 //   warp 13     work scheduler and TMA producer: takes the next work item from a global
-//               counter, publishes it to the other roles, loads its two Q tiles, then streams
-//               K/V tiles through a 4-slot ring that runs on across items
+//               counter, decodes it once into shared memory for the other roles (the decode is
+//               a dozen integer divisions), loads its two Q tiles, then streams K/V tiles
+//               through a 4-slot ring that runs on across items
 // The kernel is persistent (one CTA per SM): while the epilogue warps write out item k, the
 // producer, the MMA warp and the softmax warps already work on item k+1.
 // TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
@@ -31,23 +32,14 @@ constexpr int kRing = 4;
 constexpr float kRescaleThresholdLog2 = 8.0f;  // rescale O only when the row maximum grew by > 2^8
 
 enum WaitId : int {
-    kWaitQ = 11, kWaitFull = 12, kWaitEmpty = 13, kWaitS = 14, kWaitAlpha = 15,
+    kWaitQ = 11, kWaitFull = 12, kWaitEmpty = 13, kWaitS = 14,
     kWaitPO = 16, kWaitPV = 17, kWaitFinal = 18, kWaitItem = 19, kWaitItemFree = 20,
     kWaitQFree = 21, kWaitOFree = 22
 };
 
 // Optional in-kernel cycle accounting (compile with -DPEVLM_PROFILE): CTA 0 accumulates the
-// cycles its MMA thread and one softmax thread spend in each wait / phase and leaves them in
-// the padding of the workspace header.
-#ifdef PEVLM_PROFILE
-#define PROF_DECL(n) long long prof_acc[n] = {}; long long prof_t = clock64();
-#define PROF_LAP(i) { const long long prof_now = clock64(); prof_acc[i] += prof_now - prof_t; prof_t = prof_now; }
-#define PROF_DUMP(base, n) if (blockIdx.x == 0) { for (int prof_i = 0; prof_i < (n); ++prof_i) p.hdr->pad[(base) + prof_i] = static_cast<int32_t>(prof_acc[prof_i] >> 4); }
-#else
-#define PROF_DECL(n)
-#define PROF_LAP(i)
-#define PROF_DUMP(base, n)
-#endif
+// cycles its MMA thread and one softmax thread of each query tile spend in each wait / phase and
+// leaves them in the padding of the workspace header.
 
 template <int D>
 struct AttnSmem {

@@ -276,3 +276,30 @@ def test_mrope_bit_exact(n, Hq, Hkv, d, sections):
     torch.cuda.synchronize()
     np.testing.assert_array_equal(to_bits(qo), oracle.rope_mrope(q, 1e6, pos3, sections))
     np.testing.assert_array_equal(to_bits(ko), oracle.rope_mrope(k, 1e6, pos3, sections))
+
+
+# ---------------------------------------------------------------- many launches: no expired wait, identical results
+
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d", [(64, 64, 40, 5, 14, 2, 128), (200, 300, 9, 17, 8, 2, 128), (0, 512, 6, 64, 28, 4, 128)])
+def test_many_launches_identical(S, B, N, Q, Hq, Hkv, d):
+    """The persistent kernel hands work out through an atomic counter, so which CTA runs which item differs from
+    launch to launch; every item's arithmetic does not.  500 layer passes: status word clear, bit-identical outputs."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    from paper_2506_19651_b200.layer import LayerBuffers, layer_forward
+    w = wl(S, B, N, Q, Hq, Hkv, d, outliers=S > 0)
+    q, k, v = (to_dev(a) for a in inputs.make_qkv(w))
+    buf = LayerBuffers(gpu_shape(w))
+    ref = None
+    for i in range(500):
+        layer_forward(buf, q, k, v)
+        if i % 100 == 99 or i == 0:
+            torch.cuda.synchronize()
+            for ws in (buf.ws_prefill, buf.ws_query):
+                st, det = pb.pevlm_read_status(ws)
+                assert st == 0, (i, st, det)
+            got = (to_bits(buf.o_video).copy(), buf.lse_video.cpu().numpy().copy(), to_bits(buf.o_question).copy())
+            if ref is None:
+                ref = got
+            for a, b in zip(got, ref):
+                np.testing.assert_array_equal(a, b)

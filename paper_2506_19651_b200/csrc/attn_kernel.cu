@@ -27,13 +27,13 @@
 
 namespace pevlm {
 
-constexpr int kAttnThreads = 512;
+constexpr int kAttnThreads = 384;
 constexpr int kRing = 4;
 constexpr float kRescaleThresholdLog2 = 8.0f;  // rescale O only when the row maximum grew by > 2^8
 
 enum WaitId : int {
     kWaitQ = 11, kWaitFull = 12, kWaitEmpty = 13, kWaitS = 14,
-    kWaitPO = 16, kWaitPV = 17, kWaitFinal = 18, kWaitItem = 19, kWaitItemFree = 20,
+    kWaitPO = 16, kWaitPV = 17, kWaitItem = 19, kWaitItemFree = 20,
     kWaitQFree = 21, kWaitOFree = 22
 };
 
@@ -211,8 +211,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     __shared__ int abort_flag;
     __shared__ int s_item[2];
     __shared__ WorkItem s_decoded[2];  // the producer decodes an item once; every role copies it from here
-    __shared__ float s_final_l[2][2][kTile];  // [item parity][slot][row]: softmax may finish a short
-    __shared__ float s_final_m[2][2][kTile];  // item while the previous item's epilogue is still running
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -223,7 +221,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
     const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144;
     const uint32_t bar_final = bar0 + 176, bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
-    constexpr int kItemConsumers = 1 + 3 * kTile;  // MMA warp + two softmax warpgroups + epilogue warpgroup
+    constexpr int kItemConsumers = 1 + 2 * kTile;  // MMA warp + two softmax warpgroups
 
     if (tid == 0) {
         abort_flag = 0;
@@ -234,7 +232,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             mbar_init(bar_q_free + 8 * i, 1);
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_po + 8 * i, kTile);
-            mbar_init(bar_final + 8 * i, kTile);
             mbar_init(bar_o_free + 8 * i, kTile);
             mbar_init(bar_o_done + 8 * i, 1);
         }
@@ -249,7 +246,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
     }
-    if (warp == 12) {
+    if (warp == 8) {
         __syncwarp();
         tmem_alloc(smem_u32(&tmem_base_slot), 512);
     }
@@ -273,10 +270,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         return w;
     };
 
-    // register budget per warpgroup: 2 x 200 (softmax) + 64 (epilogue) + 48 (TMA/MMA) = 512 x 128
-    if (warp >= 12) {
-        reg_dealloc<48>();
-      if (warp == 13) {
+    // register budget per warpgroup: 2 x 216 (softmax + epilogue) + 56 (TMA/MMA) <= 384 x 168
+    if (warp >= 8) {
+        reg_dealloc<56>();
+      if (warp == 9) {
         // ------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
             int ring_idx = 0;          // K/V tiles loaded so far (ring position), runs on across items
@@ -321,7 +318,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 }
             }
         }
-      } else if (warp == 12) {
+      } else if (warp == 8) {
         // ------------------------------------------------------------- MMA issuer
         // All 32 lanes run this loop with warp-uniform values (descriptors and addresses stay in
         // uniform registers); the MMA and commit instructions themselves go out from one elected lane.
@@ -446,9 +443,9 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         }
 #endif
       }
-    } else if (warp < 8) {
-        // ------------------------------------------------------------- softmax of slot x
-        reg_alloc<200>();
+    } else {
+        // ------------------------------------------------------------- softmax and epilogue of slot x
+        reg_alloc<216>();
         const int x = warp >> 2;
         const int row = tid & 127;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -470,7 +467,22 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             const int nt = x ? it.s[1].nt : it.s[0].nt;
             const int item_ring_base = ring_base;
             ring_base += 2 * max(it.s[0].nt, it.s[1].nt);
-            if (nt == 0) continue;
+            const QSlot& qs = x ? it.s[1] : it.s[0];
+            if (!qs.valid) continue;
+            // this thread's row of the query tile
+            const bool row_ok = (row / qs.row_div < qs.ntok) && (row % qs.row_div < qs.nheads);
+            const int tok = qs.q_tok0 + row / qs.row_div;
+            const int head = qs.q_head0 + row % qs.row_div;
+            if (nt == 0) {
+                // question-mode tile with no visible key in this CTA's key range: neutral partial
+                if (p.mode == 1 && row_ok) {
+                    const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                    p.part_lse[r] = -INFINITY;
+                    float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+                    for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                continue;
+            }
             const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
             const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
             const int na = it.na, a_end = it.a_end, b_start = it.b_start;
@@ -577,73 +589,26 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
 #endif
                 l_run = l_run * alpha + sum;
             }
-            // A one-tile item never waits for the previous item's epilogue on its way here: hold the
-            // `final` arrival until that epilogue has consumed the previous one (it signals o_free after
-            // reading it), so the barrier never runs two phases ahead of its waiter.
-            if (uses > 0) wait(bar_o_free + 8 * x, (uses - 1) & 1, kWaitOFree);
-            s_final_l[uses & 1][x][row] = l_run;
-            s_final_m[uses & 1][x][row] = m_ref;
-            mbar_arrive(bar_final + 8 * x);
-            ++uses;
-        }
-#ifdef PEVLM_PROFILE
-        if ((tid == 0 || tid == 128) && blockIdx.x == 0) {
-            p.hdr->pad[8 + 8 * x] = static_cast<int32_t>(prof_busy >> 4);
-            p.hdr->pad[9 + 8 * x] = static_cast<int32_t>(prof_wait >> 4);
-            p.hdr->pad[10 + 8 * x] = static_cast<int32_t>(prof_tiles);
-            p.hdr->pad[11 + 8 * x] = static_cast<int32_t>(prof_ld >> 4);
-            p.hdr->pad[12 + 8 * x] = static_cast<int32_t>(prof_exp >> 4);
-        }
-#endif
-    } else {
-        // ------------------------------------------------------------- epilogue
-        reg_dealloc<64>();
-        const int row = tid & 127;
-        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        int uses[2] = {0, 0};   // items in which the slot was active so far (phase of final / o_done / o_free)
-        for (int k = 0;; ++k) {
-            WorkItem it;
-            const int w = next_item(k, it);
-            if (w < 0) break;
+            // Epilogue, by the same thread (its registers are free now and it would only wait for the next
+            // item's scores): once the last PV has landed, the whole accumulator row goes to registers in one
+            // round trip and the accumulator is released for the next item; normalisation, conversion and the
+            // stores follow while the next item's first QK is already in the tensor pipe.
+            wait(bar_o_done + 8 * x, uses & 1, kWaitPV);
+            tc_fence_after_sync();
+            {
+                uint32_t o[D];
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const QSlot& s = it.s[x];
-                if (!s.valid) continue;
-                const bool row_ok = (row / s.row_div < s.ntok) && (row % s.row_div < s.nheads);
-                const int tok = s.q_tok0 + row / s.row_div;
-                const int head = s.q_head0 + row % s.row_div;
-                if (s.nt == 0) {
-                    // question-mode slot with no visible key in this CTA's key range: neutral partial
-                    if (p.mode == 1 && row_ok) {
-                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-                        p.part_lse[r] = -INFINITY;
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
-                        for (int c = 0; c < D / 4; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    continue;
-                }
-                wait(bar_final + 8 * x, uses[x] & 1, kWaitFinal);
-                const float l = s_final_l[uses[x] & 1][x][row], m = s_final_m[uses[x] & 1][x][row];
-                wait(bar_o_done + 8 * x, uses[x] & 1, kWaitPV);
-                tc_fence_after_sync();
-                const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
-                const float lse_val = (l > 0.f) ? m * p.scale + logf(l) : -INFINITY;
-                const uint32_t tO = tmem_base + 256 + x * 128 + lane_off;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_wait_ld();
-                    if (c == D / 32 - 1) {
-                        // every column of this row is in registers: the accumulator may be reused
-                        tc_fence_before_sync();
-                        mbar_arrive(bar_o_free + 8 * x);
-                    }
-                    if (!row_ok) continue;
+                for (int c = 0; c < D / 32; ++c) tmem_ld32(tO + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&o[32 * c]));
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                mbar_arrive(bar_o_free + 8 * x);
+                const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+                const float lse_val = (l_run > 0.f) ? m_ref * p.scale + logf(l_run) : -INFINITY;
+                if (row_ok) {
                     if (p.mode == 0) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D + c * 32);
+                        uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D);
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
+                        for (int v = 0; v < D / 8; ++v) {
                             uint32_t wd[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
@@ -651,31 +616,33 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                                                     __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
                             dst[v] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                         }
-                    } else {
-                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D + c * 32);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
-                                                 __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
-                    }
-                }
-                if (row_ok) {
-                    if (p.mode == 0) {
                         if (p.lse) p.lse[static_cast<size_t>(head) * p.q_rows + tok] = lse_val;
                     } else {
-                        p.part_lse[(static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head] = lse_val;
+                        const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+#pragma unroll
+                        for (int v = 0; v < D / 4; ++v)
+                            dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
+                                                 __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                        p.part_lse[r] = lse_val;
                     }
                 }
             }
-#pragma unroll
-            for (int x = 0; x < 2; ++x)
-                if (it.s[x].nt > 0) ++uses[x];
+            ++uses;
         }
+#ifdef PEVLM_PROFILE
+        if ((tid & 127) == 0 && blockIdx.x == 0) {
+            p.hdr->pad[8 + 8 * x] = static_cast<int32_t>(prof_busy >> 4);
+            p.hdr->pad[9 + 8 * x] = static_cast<int32_t>(prof_wait >> 4);
+            p.hdr->pad[10 + 8 * x] = static_cast<int32_t>(prof_tiles);
+            p.hdr->pad[11 + 8 * x] = static_cast<int32_t>(prof_ld >> 4);
+            p.hdr->pad[12 + 8 * x] = static_cast<int32_t>(prof_exp >> 4);
+        }
+#endif
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 12) {
+    if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }

@@ -2,23 +2,25 @@
 //
 // One CTA owns TWO query tiles of 128 rows that share a kv head and a key-tile list (two q
 // heads of one GQA group at the same block position, or two neighbouring positions), so every
-// K/V tile staged in shared memory feeds both.  Roles (16 warps):
-//   warps 0-3   softmax of query tile 0: one thread per row; the 128 scores of a key tile are
-//               read from TMEM once, running max/sum kept in fp32, probabilities written back
-//               over the scores as bf16; the rare rescale of the O accumulator (the reference
-//               maximum moves only when a row's maximum grows by more than 2^8) is done in
-//               place by the same threads
-//   warps 4-7   softmax of query tile 1
-//   warps 8-11  epilogue: normalised output and LSE of a finished item, TMEM -> global
-//   warp 12     issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
+// K/V tile staged in shared memory feeds both.  Roles (12 warps):
+//   warps 0-3   softmax and epilogue of query tile 0: one thread per row; the 128 scores of a key
+//               tile are read from TMEM once, running max/sum kept in fp32, probabilities written
+//               back over the scores as bf16; the rare rescale of the O accumulator (the reference
+//               maximum moves only when a row's maximum grows by more than 2^8) is done in place
+//               by the same threads.  After the item's last key tile the same thread reads its
+//               row of the accumulator in one round trip, releases the accumulator, and writes
+//               the normalised output and the LSE
+//   warps 4-7   the same for query tile 1
+//   warp 8      issues the tcgen05 MMAs: S = Q K^T (both operands from shared memory) and
 //               O += P V (P from TMEM, V from shared memory), ping-ponging between the two
 //               query tiles so one is in the tensor cores while the other is in its softmax
-//   warp 13     work scheduler and TMA producer: takes the next work item from a global
+//   warp 9      work scheduler and TMA producer: takes the next work item from a global
 //               counter, decodes it once into shared memory for the other roles (the decode is
 //               a dozen integer divisions), loads its two Q tiles, then streams K/V tiles
 //               through a 4-slot ring that runs on across items
-// The kernel is persistent (one CTA per SM): while the epilogue warps write out item k, the
-// producer, the MMA warp and the softmax warps already work on item k+1.
+//   warps 10-11 idle (they complete the third warpgroup for the register reallocation)
+// The kernel is persistent (one CTA per SM): while the softmax threads write out item k, the
+// producer and the MMA warp already work on item k+1.
 // TMEM (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
 // Every wait is bounded; an expired wait records PEVLM_ETIMEOUT and the CTA still runs to its
 // normal end (waits become short), so TMEM is always released.
@@ -205,7 +207,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     extern __shared__ uint8_t smem_raw[];
     // barrier map (uint64 each): [0,2) item_full [2,4) item_free [4,6) q_full [6,8) q_free
     // [8,12) ring full [12,16) ring empty, then per slot x: [16,18) s_full [18,20) po
-    // [22,24) final [24,26) o_free [26,28) o_done
+    // [24,26) o_free [26,28) o_done
     __shared__ uint64_t bars[28];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -220,7 +222,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     const uint32_t bar_item_full = bar0, bar_item_free = bar0 + 16, bar_q_full = bar0 + 32, bar_q_free = bar0 + 48;
     const uint32_t bar_full = bar0 + 64, bar_empty = bar0 + 96;
     const uint32_t bar_s_full = bar0 + 128, bar_po = bar0 + 144;
-    const uint32_t bar_final = bar0 + 176, bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
+    const uint32_t bar_o_free = bar0 + 192, bar_o_done = bar0 + 208;
     constexpr int kItemConsumers = 1 + 2 * kTile;  // MMA warp + two softmax warpgroups
 
     if (tid == 0) {

@@ -608,24 +608,28 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 const float lse_val = (l_run > 0.f) ? m_ref * p.scale + logf(l_run) : -INFINITY;
                 if (row_ok) {
                     if (p.mode == 0) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(tok) * p.Hq + head) * D);
+                        // 32 bytes per store: every lane writes whole sectors of its own row
+                        __nv_bfloat16* dst = p.o + (static_cast<size_t>(tok) * p.Hq + head) * D;
 #pragma unroll
-                        for (int v = 0; v < D / 8; ++v) {
-                            uint32_t wd[4];
+                        for (int v = 0; v < D / 16; ++v) {
+                            uint32_t wd[8];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                wd[e] = pack_bf16x2(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
-                                                    __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
-                            dst[v] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                            for (int e = 0; e < 8; ++e)
+                                wd[e] = pack_bf16x2(__uint_as_float(o[v * 16 + 2 * e]) * inv_l,
+                                                    __uint_as_float(o[v * 16 + 2 * e + 1]) * inv_l);
+                            st_global_v8(dst + v * 16, wd);
                         }
                         if (p.lse) p.lse[static_cast<size_t>(head) * p.q_rows + tok] = lse_val;
                     } else {
                         const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + r * D);
+                        float* dst = p.part_o + r * D;
 #pragma unroll
-                        for (int v = 0; v < D / 4; ++v)
-                            dst[v] = make_float4(__uint_as_float(o[v * 4]) * inv_l, __uint_as_float(o[v * 4 + 1]) * inv_l,
-                                                 __uint_as_float(o[v * 4 + 2]) * inv_l, __uint_as_float(o[v * 4 + 3]) * inv_l);
+                        for (int v = 0; v < D / 8; ++v) {
+                            uint32_t wd[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) wd[e] = __float_as_uint(__uint_as_float(o[v * 8 + e]) * inv_l);
+                            st_global_v8(dst + v * 8, wd);
+                        }
                         p.part_lse[r] = lse_val;
                     }
                 }

@@ -74,9 +74,19 @@ struct WorkItem {
 // Optional time stamps (-DPEVLM_TRACE): clock64 at the hand-offs of CTA 0's first work item, key tiles
 // [kTraceJ0, kTraceJ0 + 16), read back through pevlm_debug_trace (see timeline.py).  Events: 0/1 scores of
 // tile 0/1 seen by the softmax, 2/3 probabilities handed over, 4 QK0 issue starts, 5 QK0 issued,
-// 6 probabilities of tile 0 seen by the MMA warp, 7 PV0 issued.
+// 6 probabilities of tile 0 seen by the MMA warp, 7 PV0 issued.  A second table holds, for CTA 0's work items
+// [kTraceK0, kTraceK0 + 16), the events of an item boundary: 0 item taken by the MMA warp, 1 its first QK goes
+// out, 2 its last PV and commits are issued; query tile 0's thread 0: 3 first scores seen, 4 last probabilities
+// handed over, 5 accumulator complete, 6 accumulator released, 7 output stored.
 #ifdef PEVLM_TRACE
 __device__ unsigned g_trace[8][16];
+__device__ unsigned g_trace_item[8][16];
+constexpr int kTraceK0 = 2;
+#define PEVLM_STAMP_ITEM(ev, kk, cond)                                                          \
+    do {                                                                                        \
+        if ((cond) && blockIdx.x == 0 && (kk) >= kTraceK0 && (kk) < kTraceK0 + 16)              \
+            g_trace_item[ev][(kk) - kTraceK0] = static_cast<unsigned>(clock64());               \
+    } while (0)
 constexpr int kTraceJ0 = 8;
 #define PEVLM_STAMP(ev, j, cond)                                                                \
     do {                                                                                        \
@@ -86,8 +96,12 @@ constexpr int kTraceJ0 = 8;
 extern "C" int pevlm_debug_trace(unsigned* host_out) {
     return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
 }
+extern "C" int pevlm_debug_trace_items(unsigned* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_trace_item, sizeof(g_trace_item)) == cudaSuccess ? 0 : -1;
+}
 #else
 #define PEVLM_STAMP(ev, j, cond) do {} while (0)
+#define PEVLM_STAMP_ITEM(ev, kk, cond) do {} while (0)
 #endif
 
 __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
@@ -339,6 +353,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_item_free + 8 * (k & 1));
             if (w < 0) break;
+            PEVLM_STAMP_ITEM(0, k, lane == 0);
             const int nt[2] = {it.s[0].nt, it.s[1].nt};
             const int nt_max = max(nt[0], nt[1]);
             // keys in the last tile of the shared range and of each slot's own range (every other
@@ -411,6 +426,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             // through the pipe without a gap.
             if (nt_max > 0) {
                 wait_full(0);
+                PEVLM_STAMP_ITEM(1, k, lane == 0);
                 if (nt[0] > 0) issue_qk(0, 0);
                 if (nt[1] > 0) issue_qk(1, 0);
                 commit_empty(0);  // K(0) consumed
@@ -430,6 +446,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 commit_empty(2 * j + 1);            // V(j) consumed
                 if (more) commit_empty(2 * j + 2);  // K(j+1) consumed
             }
+            PEVLM_STAMP_ITEM(2, k, lane == 0);
             ring_base += 2 * nt_max;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
@@ -472,9 +489,12 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             const QSlot& qs = x ? it.s[1] : it.s[0];
             if (!qs.valid) continue;
             // this thread's row of the query tile
-            const bool row_ok = (row / qs.row_div < qs.ntok) && (row % qs.row_div < qs.nheads);
-            const int tok = qs.q_tok0 + row / qs.row_div;
-            const int head = qs.q_head0 + row % qs.row_div;
+            // (row_div is 1 for all but packed tiles: no integer division on the way to the item's first scores)
+            const int row_tok = qs.row_div == 1 ? row : row / qs.row_div;
+            const int row_head = qs.row_div == 1 ? 0 : row - row_tok * qs.row_div;
+            const bool row_ok = (row_tok < qs.ntok) && (row_head < qs.nheads);
+            const int tok = qs.q_tok0 + row_tok;
+            const int head = qs.q_head0 + row_head;
             if (nt == 0) {
                 // question-mode tile with no visible key in this CTA's key range: neutral partial
                 if (p.mode == 1 && row_ok) {
@@ -488,7 +508,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             const int limit0 = x ? it.s[1].limit0 : it.s[0].limit0;
             const int b_end = x ? it.s[1].b_end : it.s[0].b_end;
             const int na = it.na, a_end = it.a_end, b_start = it.b_start;
-            const int my_limit = limit0 + row / (x ? it.s[1].row_div : it.s[0].row_div);
+            const int my_limit = limit0 + row_tok;
             float m_ref = -INFINITY;  // reference maximum (raw score units) the probabilities are scaled by
             float l_run = 0.f;
             for (int j = 0; j < nt; ++j, ++cnt) {
@@ -501,6 +521,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 prof_wait += prof_t1 - prof_t2;
 #endif
                 PEVLM_STAMP(0 + x, j, (tid & 127) == 0);
+                PEVLM_STAMP_ITEM(3, k, tid == 0 && j == 0);
                 tc_fence_after_sync();
                 // all 128 scores of the row in registers: one round trip to TMEM
                 uint32_t r[kTile];
@@ -584,6 +605,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 tc_fence_before_sync();
                 mbar_arrive(my_po);
                 PEVLM_STAMP(2 + x, j, (tid & 127) == 0);
+                PEVLM_STAMP_ITEM(4, k, tid == 0 && j == nt - 1);
 #ifdef PEVLM_PROFILE
                 prof_t2 = static_cast<unsigned>(clock64());
                 prof_busy += prof_t2 - prof_t1;
@@ -596,6 +618,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             // round trip and the accumulator is released for the next item; normalisation, conversion and the
             // stores follow while the next item's first QK is already in the tensor pipe.
             wait(bar_o_done + 8 * x, uses & 1, kWaitPV);
+            PEVLM_STAMP_ITEM(5, k, tid == 0);
             tc_fence_after_sync();
             {
                 uint32_t o[D];
@@ -604,6 +627,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 tmem_wait_ld();
                 tc_fence_before_sync();
                 mbar_arrive(bar_o_free + 8 * x);
+                PEVLM_STAMP_ITEM(6, k, tid == 0);
                 const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
                 const float lse_val = (l_run > 0.f) ? m_ref * p.scale + logf(l_run) : -INFINITY;
                 if (row_ok) {
@@ -634,6 +658,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     }
                 }
             }
+            PEVLM_STAMP_ITEM(7, k, tid == 0);
             ++uses;
         }
 #ifdef PEVLM_PROFILE

@@ -5,7 +5,8 @@
 Runs the prefill attention in full-causal mode on c3_long-sized random tensors (long work items) with a library
 built with time stamps, and prints, for 16 consecutive key tiles of CTA 0's first work item, the SM-clock
 cycles between the hand-offs of the two query tiles: scores seen by the softmax, probabilities handed to the
-MMA warp, PV and QK issue.  Rebuild without PEVLM_TRACE afterwards.
+MMA warp, PV and QK issue.  Then the same launch under the PEVLM mask (c3_long and the 256-token blocks of the
+sweep): the events at the boundaries between CTA 0's work items.  Rebuild without PEVLM_TRACE afterwards.
 """
 from __future__ import annotations
 
@@ -50,6 +51,42 @@ def main():
     print("QK issued -> scores seen by the softmax:", med((t[0] - t[5])[1:]))
     print("chain: probabilities handed over -> next scores seen:", med(t[0, 1:] - t[2, :-1]),
           " (tensor work in it: PV 512 + QK 512)")
+    del q, k, v, o, lse
+    for name in ("c3_long", "c4_sweep_F1"):
+        item_boundaries(name)
+
+
+def item_boundaries(name):
+    import torch
+    from . import binding as pb, inputs
+    w = inputs.WORKLOADS[name]
+    s = pb.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d, theta=w.theta)
+    nv = w.n_video
+    q = torch.randn(nv, w.Hq, w.d, device="cuda", dtype=torch.bfloat16)
+    k = torch.randn(nv, w.Hkv, w.d, device="cuda", dtype=torch.bfloat16)
+    v = torch.randn_like(k)
+    o = torch.empty_like(q)
+    lse = torch.empty(w.Hq, nv, device="cuda")
+    ws = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        pb.pevlm_parallel_prefill_attn(s, q, k, v, o, lse, ws)
+    torch.cuda.synchronize()
+    buf = (C.c_uint32 * 128)()
+    assert pb.lib().pevlm_debug_trace_items(buf) == 0
+    t = np.array(buf, dtype=np.int64).reshape(8, 16)[:, :12]   # items 2..13 of CTA 0
+
+    def med(a):
+        return int(np.median(a & 0xFFFFFFFF))
+    print(f"-- work-item boundaries, {name} under the PEVLM mask (medians over 11-12 items of CTA 0, cycles)")
+    print("item (first scores seen -> next item's first scores seen):", med(t[3, 1:] - t[3, :-1]))
+    print("last probabilities of tile 0 handed over -> accumulator complete:", med(t[5] - t[4]))
+    print("accumulator complete -> released:", med(t[6] - t[5]))
+    print("released -> output stored:", med(t[7] - t[6]))
+    print("last probabilities of tile 0 -> MMA warp has issued the item's last PV and commits:", med(t[2] - t[4]))
+    print("MMA warp: end of item -> next item taken:", med(t[0, 1:] - t[2, :-1]))
+    print("next item taken -> its first QK goes out:", med(t[1] - t[0]))
+    print("first QK goes out -> first scores seen:", med(t[3] - t[1]))
+    print("last probabilities of tile 0 -> next item's first scores seen:", med(t[3, 1:] - t[4, :-1]))
 
 
 if __name__ == "__main__":

@@ -643,7 +643,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                                                     __uint_as_float(o[v * 16 + 2 * e + 1]) * inv_l);
                             st_global_v8(dst + v * 16, wd);
                         }
-                        if (p.lse) p.lse[static_cast<size_t>(head) * p.q_rows + tok] = lse_val;
+                        if (p.lse) st_global_stream_f32(p.lse + static_cast<size_t>(head) * p.q_rows + tok, lse_val);
                     } else {
                         const size_t r = (static_cast<size_t>(it.split) * p.Q + tok) * p.Hq + head;
                         float* dst = p.part_o + r * D;
@@ -654,7 +654,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                             for (int e = 0; e < 8; ++e) wd[e] = __float_as_uint(__uint_as_float(o[v * 8 + e]) * inv_l);
                             st_global_v8(dst + v * 8, wd);
                         }
-                        p.part_lse[r] = lse_val;
+                        st_global_stream_f32(p.part_lse + r, lse_val);
                     }
                 }
             }

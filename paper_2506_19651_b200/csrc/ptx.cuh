@@ -323,6 +323,10 @@ __device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&w)[8]) 
                  : "memory");
 }
 
+__device__ __forceinline__ void st_global_stream_f32(float* ptr, float v) {
+    asm volatile("st.global.L1::no_allocate.f32 [%0], %1;" ::"l"(ptr), "f"(v) : "memory");
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

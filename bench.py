@@ -30,7 +30,7 @@ from paper_2506_19651_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pevlm_parallel_prefill_attn launch, from the
 # ncu captures summarised in profiles/attn_kernel_c3_long_c5_stack_ncu_metrics.md (and the c2_qwen full capture)
-NCU_PREFILL_TRAFFIC_BYTES = {"c3_long": 794.7e6, "c5_stack": 1184.9e6, "c2_qwen": 173.4e6}
+NCU_PREFILL_TRAFFIC_BYTES = {"c3_long": 793.0e6, "c5_stack": 1181.3e6, "c2_qwen": 173.4e6}
 
 METRIC = "active_tile_tflops_per_layer"
 UNIT = "TFLOP/s"

@@ -260,6 +260,17 @@ __device__ __forceinline__ void mma_ts_batch4(uint32_t d_tmem, uint32_t a_tmem, 
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate_first));
 }
 
+// Same over 32 keys (two steps).
+__device__ __forceinline__ void mma_ts_batch2(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t accumulate_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b32 ta, tb;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        PEVLM_MMA_TS_STEP(0, 0, "p0") PEVLM_MMA_TS_STEP(8, 128, "p1")
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate_first));
+}
+
 // Same over 128 keys (eight steps).
 __device__ __forceinline__ void mma_ts_batch8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
                                               uint32_t accumulate_first) {

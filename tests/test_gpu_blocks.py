@@ -141,3 +141,48 @@ def test_streaming_window(S, B, W, T, Q, Hq, Hkv, d):
     assert np.abs(lse_q.double().cpu().numpy().T - lse).max() <= LSE_TOL
     # the cache holds exactly those roped keys
     np.testing.assert_array_equal(to_bits(win.k_cache[:S + held * B + Q]), kr[idx])
+
+
+def test_sequences_of_different_shapes_share_one_cache_buffer():
+    """Per-sequence shapes: three streams with different (S, B, N, Q) packed back to back in one K/V cache buffer,
+    one group of calls per stream on slices of the shared buffers, all on one CUDA stream without a sync in between."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    Hq, Hkv, d, theta = 8, 2, 128, 1e6
+    seqs = [(64, 128, 3, 8), (96, 160, 2, 5), (0, 256, 2, 4)]
+    ws_list, outs, streams = [], [], []
+    total = sum(S + N * B + Q for S, B, N, Q in seqs)
+    k_cache = torch.zeros((total, Hkv, d), dtype=torch.bfloat16, device="cuda")
+    v_cache = torch.zeros_like(k_cache)
+    row = 0
+    for i, (S, B, N, Q) in enumerate(seqs):
+        w = inputs.Workload("t", S, B, N, Q, Hq, Hkv, d, theta, S > 0, 900 + i)
+        q, k, v = inputs.make_qkv(w)
+        streams.append((w, q, k, v))
+        s = pb.make_shape(S, B, N, Q, Hq, Hkv, d, theta=theta)
+        nv, L = w.n_video, w.L
+        kc, vc = k_cache[row:row + L], v_cache[row:row + L]
+        qd = to_dev(q)
+        pb.pevlm_rope_qk(s, qd, to_dev(k), qd, kc, 0, L)
+        pb.pevlm_assemble_kv(s, None, to_dev(v[:nv]), None, to_dev(v[nv:]), kc, vc)
+        o_v = torch.empty((nv, Hq, d), dtype=torch.bfloat16, device="cuda")
+        lse_v = torch.empty((Hq, nv), dtype=torch.float32, device="cuda")
+        o_q = torch.empty((Q, Hq, d), dtype=torch.bfloat16, device="cuda")
+        lse_q = torch.empty((Hq, Q), dtype=torch.float32, device="cuda")
+        ws_p = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device="cuda")
+        ws_q = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device="cuda")
+        pb.pevlm_parallel_prefill_attn(s, qd[:nv], kc[:nv], vc[:nv], o_v, lse_v, ws_p)
+        pb.pevlm_query_attn(s, qd[nv:], kc, vc, o_q, lse_q, ws_q)
+        ws_list += [ws_p, ws_q]
+        outs.append((o_v, lse_v, o_q, lse_q))
+        row += L
+    torch.cuda.synchronize()
+    _status_ok(*ws_list)
+    for (w, q, k, v), (o_v, lse_v, o_q, lse_q) in zip(streams, outs):
+        qr, kr = oracle.rope(q, theta), oracle.rope(k, theta)
+        sh = oracle.make_shape(w.S, w.B, w.N, w.Q, Hq, Hkv, d)
+        o, lse = oracle.attn_rows(sh, qr, kr, v, np.arange(w.L, dtype=np.int64))
+        o_gpu = np.concatenate([bits_to_f64(to_bits(o_v)), bits_to_f64(to_bits(o_q))])
+        lse_gpu = np.concatenate([lse_v.double().cpu().numpy().T, lse_q.double().cpu().numpy().T])
+        assert np.abs(o_gpu - o).max() <= O_TOL
+        assert np.abs(lse_gpu - lse).max() <= LSE_TOL

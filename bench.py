@@ -257,11 +257,13 @@ def run_ours(args, w):
     clocks = sampler.stop() if sampler else None
     ms_total = max_over_ranks(t_begin.elapsed_time(t_end))
     ms_step = ms_total / args.steps
-    per_kernel = {n: 0.0 for n in names}
+    samples = {n: [] for n in names}
     for (n0, e0), (n1, e1) in zip(marks[:-1], marks[1:]):
         if n1 != "start":
-            per_kernel[n1] += e0.elapsed_time(e1)
-    per_kernel = {n: t / args.steps for n, t in per_kernel.items()}
+            samples[n1].append(e0.elapsed_time(e1))
+    per_kernel = {n: sum(t) / args.steps for n, t in samples.items()}
+    prefill_spread = {"ms_median": statistics.median(samples["prefill_attn"]), "ms_min": min(samples["prefill_attn"]),
+                      "ms_max": max(samples["prefill_attn"])} if samples.get("prefill_attn") else {}
     for ws in (buf.ws_prefill, buf.ws_query):
         st, det = pb.pevlm_read_status(ws)
         if st != 0:
@@ -338,7 +340,8 @@ def run_ours(args, w):
         "kernels_ms": per_kernel,
         "prefill": {"ms": t_pre, "active_tile_tflops": achieved, "useful_tflops": useful_prefill / (t_pre * 1e-3) / 1e12,
                     "active_tiles": pre.tiles, "frac_of_bf16_peak": achieved / peaks["bf16_tflops"],
-                    "frac_of_bf16_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None},
+                    "frac_of_bf16_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
+                    **prefill_spread},
         "query": {"ms": per_kernel["query_attn"], "active_tile_tflops": que.flops / (per_kernel["query_attn"] * 1e-3) / 1e12,
                   "cache_gbs": kv_bytes / (per_kernel["query_attn"] * 1e-3) / 1e9},
         "assemble": {"ms": per_kernel["assemble_video"], "gbs": 2.0 * w.n_video * w.Hkv * w.d * 2 / (per_kernel["assemble_video"] * 1e-3) / 1e9},

@@ -41,6 +41,8 @@ def lib():
         _lib.oracle_num_threads.restype = C.c_int
         _lib.oracle_visible.restype = C.c_int
         _lib.oracle_count_pairs.restype = C.c_int64
+        _lib.oracle_round_bf16.restype = C.c_uint16
+        _lib.oracle_round_bf16.argtypes = [C.c_double]
         _lib.oracle_count_rect_pairs.restype = C.c_int64
     return _lib
 
@@ -57,6 +59,11 @@ def _u16(a):
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def round_bf16(x: float) -> int:
+    """bf16 bit pattern of the two-step rounding fp64 -> fp32 -> bf16 (both to nearest even) the RoPE ends with."""
+    return int(lib().oracle_round_bf16(float(x)))
 
 
 def visible(sh: Shape, t: int):

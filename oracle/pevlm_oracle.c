@@ -32,8 +32,9 @@
  * sink rows == full-attention rows, softmax weights sum to 1, block-permutation
  * invariance with carried positions, closed forms with K = 0 (LSE = ln #visible,
  * O = prefix mean of V), Eq. 10's pair count, RoPE closed forms (position 0 identity,
- * norm preservation, relative-position property), merge == unsplit, and a literal
- * pure-Python triple loop on tiny shapes.
+ * norm preservation, relative-position property), the bf16 rounding on hand-worked bit
+ * patterns (round up, round down, ties to even both ways, the two-step case), merge ==
+ * unsplit, and a literal pure-Python triple loop on tiny shapes.
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see oracle/build.py).
  */
@@ -76,6 +77,9 @@ static uint16_t f64_to_bf16(double x) {
     u += 0x7FFFu + lsb;
     return (uint16_t)(u >> 16);
 }
+
+/* The rounding R1 as a scalar, so that it can be pinned with hand-worked bit patterns. */
+uint16_t oracle_round_bf16(double x) { return f64_to_bf16(x); }
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP

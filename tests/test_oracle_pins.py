@@ -281,6 +281,50 @@ def test_p7_bf16_rounding_is_nearest_even():
     assert _bf16_bits_of(1 + 2 ** -8) == 0x3F80 and _bf16_bits_of(1 + 3 * 2 ** -8) == 0x3F82
 
 
+# R1, the one rounding of the oracle (fp64 -> fp32 -> bf16, both to nearest even), pinned on bit patterns
+# worked out by hand from the binary expansions; the comments give the fp32 word before the second step.
+R1_HAND = [
+    (0.3, 0x3E9A),                        # 0x3E99999A: low half 0x999A > 0x8000, rounds UP
+    (-0.3, 0xBE9A),                       # sign does not change the magnitude rounding
+    (1 + 2.0 ** -9, 0x3F80),              # 0x3F804000: below half, rounds down
+    (1 + 2.0 ** -8, 0x3F80),              # 0x3F808000: exact tie, 0x3F80 is even, stays
+    (1 + 3 * 2.0 ** -8, 0x3F82),          # 0x3F818000: exact tie, 0x3F81 is odd, goes up to even
+    (-(1 + 3 * 2.0 ** -8), 0xBF82),
+    (1 + 2.0 ** -8 + 2.0 ** -20, 0x3F81),  # 0x3F808008: just above the tie, rounds up
+    (1 + 2.0 ** -8 + 2.0 ** -30, 0x3F80),  # two steps: fp32 drops 2^-30 (tie 0x3F808000 -> even); one step would give 0x3F81
+    (1 + 2.0 ** -7 - 2.0 ** -30, 0x3F81),  # fp32 rounds up to 0x3F810000 exactly: 0x3F81
+    (1 + 3 * 2.0 ** -8 - 2.0 ** -30, 0x3F82),  # fp32 gives the tie 0x3F818000 -> even 0x3F82; one step would give 0x3F81
+    (0.0, 0x0000), (1.0, 0x3F80), (-2.0, 0xC000), (3.140625, 0x4049),
+    (65280.0, 0x477F), (65408.0, 0x4780),  # 0x477F8000: tie with odd upper half, carries into the exponent
+]
+
+
+@pytest.mark.parametrize("x,bits", R1_HAND)
+def test_r1_rounding_hand_values(x, bits):
+    assert api.round_bf16(x) == bits
+
+
+def test_r1_rounding_through_rope_matches_fp64_output():
+    # the bits the RoPE emits are the scalar rounding of the fp64 values it reports, and both agree with an
+    # independent integer formulation of the two-step rounding, on a few thousand roped elements
+    w = inputs.Workload("t", 40, 1, 0, 0, 3, 3, 32, 1e6, False, 77)
+    q, _, _ = inputs.make_qkv(w)
+    out, f64 = api.rope(q, 1e6, first_pos=50000, want_f64=True)
+    flat_bits, flat = out.reshape(-1), f64.reshape(-1)
+    assert flat.size >= 3000
+    f32_words = flat.astype(np.float32).view(np.uint32).astype(np.uint64)    # step 1 by numpy's cast (RNE)
+    low, upper = f32_words & 0xFFFF, f32_words >> 16
+    up = (low > 0x8000) | ((low == 0x8000) & ((upper & 1) == 1))             # step 2 spelled out as a comparison
+    expect = ((upper + up.astype(np.uint64)) & 0xFFFF).astype(np.uint16)
+    np.testing.assert_array_equal(flat_bits, expect)
+    assert up.sum() > 1000 and (~up).sum() > 1000                           # both directions occur
+    for i in range(0, flat.size, 97):
+        assert api.round_bf16(float(flat[i])) == int(flat_bits[i])
+    # position 0 is the identity on fp64, so bf16 inputs come back bit for bit (no rounding error at all)
+    mrope_bits = api.rope_mrope(q, 1e6, np.zeros((3, 40), dtype=np.int64), (4, 6, 6))
+    np.testing.assert_array_equal(mrope_bits, q)
+
+
 def test_p7_rope_position_zero_identity_and_norm():
     w = inputs.Workload("t", 16, 1, 0, 0, 3, 3, 16, 1e6, False, 9)
     q, _, _ = inputs.make_qkv(w)

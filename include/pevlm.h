@@ -15,12 +15,18 @@
  * natural log of the sum of exp(scaled score).
  *
  * General rules for every entry point
- *   - All tensor pointers are DEVICE pointers, 16-byte aligned, contiguous, bf16
- *     (2-byte brain float) unless stated.  `stream` is a cudaStream_t passed as void*
- *     (NULL = the legacy default stream).  `shape` is a HOST pointer.
+ *   - All tensor pointers are DEVICE pointers, contiguous, bf16 (2-byte brain float) unless
+ *     stated, and 16-byte aligned; the attention OUTPUT `o` of pevlm_parallel_prefill_attn,
+ *     pevlm_block_attn and pevlm_query_attn(_noalloc) must be 32-byte aligned (its rows are
+ *     written with 32-byte vector stores), workspaces 256-byte aligned.  A pointer that misses
+ *     its alignment is refused with PEVLM_EALIGN before any launch.  `stream` is a
+ *     cudaStream_t passed as void* (NULL = the legacy default stream).  `shape` is a HOST
+ *     pointer.  Input values must be finite.
  *   - The caller owns every buffer and the stream.  The library allocates no device
- *     memory, keeps no state between calls, never synchronises the device and never
- *     frees anything.  Calls are asynchronous on `stream`.
+ *     memory, never synchronises the device (pevlm_read_status excepted) and never frees
+ *     anything.  Calls are asynchronous on `stream`.  No state is kept between calls, with
+ *     one exception: pevlm_query_attn_noalloc owns a fixed device array per GPU and
+ *     remembers its address (see there).
  *   - batch > 1 means `batch` independent sequences of the same shape, stored one after
  *     another (the leading dimension of every tensor, and of the workspace partials).
  *   - Return value: PEVLM_OK (0) or a negative pevlm_status_t.  All argument checking
@@ -41,7 +47,7 @@ extern "C" {
 typedef enum {
     PEVLM_OK = 0,
     PEVLM_EINVAL = -1,       /* bad shape or NULL pointer */
-    PEVLM_EALIGN = -2,       /* a pointer is not 16-byte aligned */
+    PEVLM_EALIGN = -2,       /* a pointer misses its alignment (16 bytes; attention outputs 32; workspaces 256) */
     PEVLM_EUNSUPPORTED = -3, /* head_dim not in {64,128}, device is not sm_100, ... */
     PEVLM_EWORKSPACE = -4,   /* workspace NULL or too small */
     PEVLM_ECUDA = -5,        /* a CUDA call failed; text via pevlm_last_cuda_error */
@@ -87,8 +93,8 @@ int pevlm_rope_qk(const pevlm_shape_t* shape, const void* q_in, const void* k_in
                   void* stream);
 
 /*
- * Multimodal RoPE, the position embedding of the Qwen2-VL family the paper evaluates ("their position
- * embeddings also incorporate spatio-temporal information", Sec. 3.1): every token has three position
+ * Multimodal RoPE: the model family the paper evaluates encodes temporal and spatial coordinates in its
+ * position embedding (Sec. 3.1), so every token has three position
  * components, pos_ids3 = device int32 [3, n_tokens] (temporal, height, width).  Rotary pair i < d/2 takes
  * its position from component 0 for i < sections[0], from component 1 for the next sections[1] pairs and
  * from component 2 for the last sections[2] (host int32[3], sum = d/2; the split itself is the model's,
@@ -125,7 +131,9 @@ int pevlm_parallel_prefill_attn(const pevlm_shape_t* shape, const void* q, const
  * future work, Sec. 5), (iii) per-sequence shapes, one call per shape.  mask_mode must be
  * PEVLM_MASK_PEVLM; first_key_row >= S and first_key_row + N*B <= cache_rows, else PEVLM_EINVAL.
  * batch strides: N*B rows for q / o / lse, cache_rows rows for the caches.  Workspace as for
- * pevlm_parallel_prefill_attn.
+ * pevlm_parallel_prefill_attn.  Only cache rows [0, S) and the block range are read: a ragged last key tile
+ * takes zeros, not the neighbouring rows, past the end of either range, so the rest of the cache may hold
+ * anything (uninitialised slots of a streaming window included).
  */
 int pevlm_block_attn(const pevlm_shape_t* shape, const void* q_blocks, const void* k_cache,
                      const void* v_cache, int64_t first_key_row, int64_t cache_rows, void* o, float* lse,
@@ -173,8 +181,8 @@ int pevlm_query_attn(const pevlm_shape_t* shape, const void* q_question, const v
  *     each call clears the status header it needs on the stream and overwrites the partials it
  *     reads.  Two calls whose kernels overlap on the GPU (different streams, no ordering
  *     between them) race on the array; order them.
- *   - A device-side timeout is left in the array's header; it cannot be read back through
- *     pevlm_read_status, which takes a caller workspace.
+ *   - A device-side timeout is left in the array's header; pevlm_read_status with
+ *     workspace = NULL reads it back (for the current device).
  */
 #define PEVLM_NOALLOC_SCRATCH_BYTES (32u << 20)
 int pevlm_query_attn_noalloc(const pevlm_shape_t* shape, const void* q_question, const void* k_cache,
@@ -184,11 +192,21 @@ int pevlm_query_attn_noalloc(const pevlm_shape_t* shape, const void* q_question,
 size_t pevlm_workspace_bytes(const pevlm_shape_t* shape, int which /* pevlm_workspace_kind_t */);
 
 /*
- * Reads the status word a kernel may have left in `workspace` (device pointer).  Blocks
- * the calling host thread until `stream` is idle.  *status = PEVLM_OK or PEVLM_ETIMEOUT;
- * *detail (may be NULL) = an implementation-defined code naming the wait that expired.
+ * Reads the status word a kernel may have left in `workspace` (device pointer; NULL = the
+ * built-in array of pevlm_query_attn_noalloc on the current device).  Blocks the calling host
+ * thread until `stream` is idle.  *status = PEVLM_OK or PEVLM_ETIMEOUT; *detail (may be NULL)
+ * = wait id * 1000000 + index of the thread block whose wait expired.
  */
 int pevlm_read_status(const void* workspace, void* stream, int32_t* status, int32_t* detail);
+
+/*
+ * Self-test of the failure path (the paper has no counterpart): launches one thread block that
+ * waits, with the library's bounded wait, on a barrier nothing ever arrives on.  After limit_ns
+ * (1 us .. 100 ms) the wait gives up, the kernel records PEVLM_ETIMEOUT with wait id 99 in the
+ * header of `workspace` (>= 256 bytes, 256-byte aligned) and ends normally; the context stays
+ * usable and the next call on the same workspace clears the status.  Nothing traps or faults.
+ */
+int pevlm_selftest_wait_expiry(void* workspace, size_t workspace_bytes, int64_t limit_ns, void* stream);
 
 /*
  * Executed tensor-core work of a call for this shape, for throughput accounting:

@@ -23,7 +23,7 @@ NOALLOC_SCRATCH_BYTES = 32 << 20
 
 EXPORTS = ["pevlm_rope_qk", "pevlm_rope_qk_mrope", "pevlm_parallel_prefill_attn", "pevlm_block_attn", "pevlm_assemble_kv", "pevlm_query_attn",
            "pevlm_query_attn_noalloc",
-           "pevlm_workspace_bytes", "pevlm_read_status", "pevlm_tile_stats", "pevlm_strerror",
+           "pevlm_workspace_bytes", "pevlm_read_status", "pevlm_selftest_wait_expiry", "pevlm_tile_stats", "pevlm_strerror",
            "pevlm_last_cuda_error"]
 
 
@@ -79,6 +79,8 @@ def lib():
         l.pevlm_workspace_bytes.argtypes = [sp, C.c_int]
         l.pevlm_workspace_bytes.restype = C.c_size_t
         l.pevlm_read_status.argtypes = [vp, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        l.pevlm_selftest_wait_expiry.argtypes = [vp, C.c_size_t, C.c_int64, vp]
+        l.pevlm_selftest_wait_expiry.restype = C.c_int
         l.pevlm_tile_stats.argtypes = [sp, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
         l.pevlm_strerror.argtypes = [C.c_int]
         l.pevlm_strerror.restype = C.c_char_p
@@ -149,7 +151,13 @@ def pevlm_query_attn_noalloc(shape: Shape, q_question, k_cache, v_cache, o, lse)
                                           _ptr(lse), _stream()), "pevlm_query_attn_noalloc")
 
 
+def pevlm_selftest_wait_expiry(workspace, limit_ns: int):
+    _check(lib().pevlm_selftest_wait_expiry(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                            limit_ns, _stream()), "pevlm_selftest_wait_expiry")
+
+
 def pevlm_read_status(workspace):
+    """workspace = None reads the built-in array of pevlm_query_attn_noalloc on the current device."""
     st, det = C.c_int32(0), C.c_int32(0)
     _check(lib().pevlm_read_status(_ptr(workspace), _stream(), C.byref(st), C.byref(det)), "pevlm_read_status")
     return st.value, det.value

@@ -14,7 +14,7 @@ import sys
 _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
 LIB = os.path.join(_DIR, "libpevlm.so")
-SOURCES = ["api.cu", "rope_kernel.cu", "assemble_kernel.cu", "attn_kernel.cu", "merge_kernel.cu", "query_noalloc.cu"]
+SOURCES = ["api.cu", "rope_kernel.cu", "assemble_kernel.cu", "attn_kernel.cu", "merge_kernel.cu", "query_noalloc.cu", "selftest.cu"]
 HEADERS = ["internal.h", "ptx.cuh", os.path.join("..", "..", "include", "pevlm.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]
@@ -36,9 +36,8 @@ def _stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    extra = ["-DPEVLM_PROFILE"] if os.environ.get("PEVLM_PROFILE") == "1" else []
-    if os.environ.get("PEVLM_TRACE") == "1":   # time stamps of the kernel's hand-offs, read by timeline.py
-        extra.append("-DPEVLM_TRACE")
+    # PEVLM_TRACE=1: time stamps of the kernel's hand-offs, read by timeline.py (include/pevlm_trace.h)
+    extra = ["-DPEVLM_TRACE"] if os.environ.get("PEVLM_TRACE") == "1" else []
     if not force and not _stale():
         return LIB
     objs = []

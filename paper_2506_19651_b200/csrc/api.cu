@@ -6,6 +6,7 @@
 #include <cstring>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace pevlm {
 
@@ -22,6 +23,7 @@ int fail_with_text(int code, const char* text) {
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
 static int check_shape(const pevlm_shape_t* s) {
@@ -149,6 +151,17 @@ static size_t query_partial_floats(const pevlm_shape_t* s, const QueryPlan& q) {
     return static_cast<size_t>(q.n_splits) * s->query_len * s->num_q_heads * (s->head_dim + 1);
 }
 
+// Host-side argument checks of the question attention, shared by its two entry points.
+int check_query_args(const pevlm_shape_t* s, const void* q_question, const void* k_cache, const void* v_cache,
+                     const void* o, const float* lse) {
+    const int rc = check_shape(s);
+    if (rc != PEVLM_OK) return rc;
+    if (!q_question || !k_cache || !v_cache || !o) return PEVLM_EINVAL;
+    if (!aligned16(q_question) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned32(o) || !aligned16(lse))
+        return PEVLM_EALIGN;
+    return PEVLM_OK;
+}
+
 }  // namespace pevlm
 
 using namespace pevlm;
@@ -159,7 +172,7 @@ const char* pevlm_strerror(int code) {
     switch (code) {
         case PEVLM_OK: return "ok";
         case PEVLM_EINVAL: return "invalid shape or NULL pointer";
-        case PEVLM_EALIGN: return "pointer not 16-byte aligned (workspace: 256-byte)";
+        case PEVLM_EALIGN: return "pointer not 16-byte aligned (attention outputs: 32-byte, workspace: 256-byte)";
         case PEVLM_EUNSUPPORTED: return "unsupported head_dim / group size, or device is not sm_100";
         case PEVLM_EWORKSPACE: return "workspace missing or too small";
         case PEVLM_ECUDA: return "CUDA error (see pevlm_last_cuda_error)";
@@ -274,7 +287,8 @@ static int prefill_common(const pevlm_shape_t* s, const void* q, const void* k, 
     int rc = check_shape(s);
     if (rc != PEVLM_OK) return rc;
     if (!q || !k || !v || !o) return PEVLM_EINVAL;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return PEVLM_EALIGN;
+    // the output rows are written with 32-byte vector stores
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned32(o) || !aligned16(lse)) return PEVLM_EALIGN;
     if (!workspace || workspace_bytes < pevlm_workspace_bytes(s, PEVLM_WS_PREFILL)) return PEVLM_EWORKSPACE;
     if (!aligned256(workspace)) return PEVLM_EALIGN;
     const int64_t nv = n_video(s);
@@ -331,25 +345,35 @@ static int prefill_common(const pevlm_shape_t* s, const void* q, const void* k, 
     p.n_items = p.items_block + p.Hkv * p.pairs_sink;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
+    p.wait_limit_ns = kDefaultWaitLimitNs;
     p.hdr = static_cast<WorkspaceHeader*>(workspace);
+    const int64_t block_rows_launch = static_cast<int64_t>(p.N) * p.B;  // full causal: the whole stream as one block
     for (int b = 0; b < s->batch; ++b) {
         const int64_t qoff = static_cast<int64_t>(b) * q_rows * p.Hq * d, koff = static_cast<int64_t>(b) * kv_rows * p.Hkv * d;
-        CUtensorMap tq, tq_tb, tq_ts, tk, tv;
+        AttnMaps m;
         const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q) + qoff;
-        if ((rc = make_tmap(&tq, qb, q_rows, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
-        tq_tb = tq;
-        tq_ts = tq;
-        if (pb.tail_tiles > 0 && (rc = make_tmap(&tq_tb, qb, q_rows, p.Hq, d, pb.tail_heads, pb.tail_rows)) != PEVLM_OK) return rc;
-        if (ps.tail_tiles > 0 && (rc = make_tmap(&tq_ts, qb, q_rows, p.Hq, d, ps.tail_heads, ps.tail_rows)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k) + koff, kv_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v) + koff, kv_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&m.q, qb, q_rows, p.Hq, d, 1, kTile)) != PEVLM_OK) return rc;
+        m.q_tail_block = m.q;
+        m.q_tail_sink = m.q;
+        if (pb.tail_tiles > 0 && (rc = make_tmap(&m.q_tail_block, qb, q_rows, p.Hq, d, pb.tail_heads, pb.tail_rows)) != PEVLM_OK) return rc;
+        if (ps.tail_tiles > 0 && (rc = make_tmap(&m.q_tail_sink, qb, q_rows, p.Hq, d, ps.tail_heads, ps.tail_rows)) != PEVLM_OK) return rc;
+        // K and V: one map over the sink rows [0, S) and one over the block rows, so that the ragged last key
+        // tile of either range reads zeros past its end (a map needs at least one row; an empty range is never read)
+        const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k) + koff;
+        const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v) + koff;
+        const int64_t blk_off = static_cast<int64_t>(p.blk_key0) * p.Hkv * d;
+        const int64_t sink_rows = p.S > 0 ? p.S : 1, blk_rows = block_rows_launch > 0 ? block_rows_launch : 1;
+        if ((rc = make_tmap(&m.k_sink, kb, sink_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&m.v_sink, vb, sink_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&m.k, kb + blk_off, blk_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&m.v, vb + blk_off, blk_rows, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
         p.o = static_cast<__nv_bfloat16*>(o) + qoff;
         p.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * q_rows : nullptr;
         if (b > 0) {  // every launch starts its work counter at zero; the status word is kept
             e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
             if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
         }
-        e = launch_attn(p, d, tq, tq_tb, tq_ts, tk, tv, st);
+        e = launch_attn(p, d, m, st);
         if (e != cudaSuccess) return cuda_fail(e, "prefill attention launch");
     }
     return PEVLM_OK;
@@ -369,11 +393,8 @@ int pevlm_block_attn(const pevlm_shape_t* s, const void* q_blocks, const void* k
 
 int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void* k_cache, const void* v_cache, void* o,
                      float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    int rc = check_shape(s);
+    int rc = check_query_args(s, q_question, k_cache, v_cache, o, lse);
     if (rc != PEVLM_OK) return rc;
-    if (!q_question || !k_cache || !v_cache || !o) return PEVLM_EINVAL;
-    if (!aligned16(q_question) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(lse))
-        return PEVLM_EALIGN;
     if (!workspace || workspace_bytes < pevlm_workspace_bytes(s, PEVLM_WS_QUERY)) return PEVLM_EWORKSPACE;
     if (!aligned256(workspace)) return PEVLM_EALIGN;
     if (s->query_len == 0) return PEVLM_OK;
@@ -401,6 +422,7 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
     p.n_items = p.Hkv * ((p.q_tiles + 1) / 2) * p.n_splits;
     p.scale = resolve_scale(s);
     p.scale_log2 = p.scale * 1.4426950408889634f;
+    p.wait_limit_ns = kDefaultWaitLimitNs;
     p.hdr = static_cast<WorkspaceHeader*>(workspace);
     const size_t part_floats = query_partial_floats(s, qp);
     const size_t part_stride = (part_floats * sizeof(float) + 255) / 256 * 256;
@@ -413,11 +435,12 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
             e = cudaMemsetAsync(&p.hdr->work_counter, 0, sizeof(int32_t), st);
             if (e != cudaSuccess) return cuda_fail(e, "work counter memset");
         }
-        CUtensorMap tq, tk, tv;
-        if ((rc = make_tmap(&tq, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tk, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        if ((rc = make_tmap(&tv, static_cast<const __nv_bfloat16*>(v_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
-        e = launch_attn(p, d, tq, tq, tq, tk, tv, st);
+        AttnMaps maps;
+        if ((rc = make_tmap(&maps.q, static_cast<const __nv_bfloat16*>(q_question) + qoff, p.Q, p.Hq, d, p.G, p.tok_per_tile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&maps.k, static_cast<const __nv_bfloat16*>(k_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        if ((rc = make_tmap(&maps.v, static_cast<const __nv_bfloat16*>(v_cache) + koff, L, p.Hkv, d, 1, kTile)) != PEVLM_OK) return rc;
+        maps.q_tail_block = maps.q; maps.q_tail_sink = maps.q; maps.k_sink = maps.k; maps.v_sink = maps.v;
+        e = launch_attn(p, d, maps, st);
         if (e != cudaSuccess) return cuda_fail(e, "question attention launch");
         MergeParams m;
         m.Q = p.Q; m.Hq = p.Hq; m.d = d; m.n_splits = p.n_splits;
@@ -430,8 +453,28 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
     return PEVLM_OK;
 }
 
+int pevlm_selftest_wait_expiry(void* workspace, size_t workspace_bytes, int64_t limit_ns, void* stream) {
+    if (!workspace || workspace_bytes < kStatusBytes) return PEVLM_EWORKSPACE;
+    if (!aligned256(workspace)) return PEVLM_EALIGN;
+    if (limit_ns < 1000 || limit_ns > 100ll * 1000 * 1000) return PEVLM_EINVAL;  // 1 us .. 100 ms
+    int rc = check_device();
+    if (rc != PEVLM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, st);
+    if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
+    e = launch_wait_selftest(static_cast<WorkspaceHeader*>(workspace), static_cast<uint64_t>(limit_ns), st);
+    if (e != cudaSuccess) return cuda_fail(e, "wait self-test launch");
+    return PEVLM_OK;
+}
+
 int pevlm_read_status(const void* workspace, void* stream, int32_t* status, int32_t* detail) {
-    if (!workspace || !status) return PEVLM_EINVAL;
+    if (!status) return PEVLM_EINVAL;
+    if (!workspace) {  // the built-in array of pevlm_query_attn_noalloc on the current device
+        void* scratch = nullptr;
+        const int rc = noalloc_scratch_for_current_device(&scratch);
+        if (rc != PEVLM_OK) return rc;
+        workspace = scratch;
+    }
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     int32_t words[2] = {0, 0};

@@ -39,10 +39,6 @@ enum WaitId : int {
     kWaitQFree = 21, kWaitOFree = 22
 };
 
-// Optional in-kernel cycle accounting (compile with -DPEVLM_PROFILE): CTA 0 accumulates the
-// cycles its MMA thread and one softmax thread of each query tile spend in each wait / phase and
-// leaves them in the padding of the workspace header.
-
 template <int D>
 struct AttnSmem {
     static constexpr int kPanels = D / 64;
@@ -66,8 +62,11 @@ struct QSlot {
     int valid;
     int q_tok0, q_head0, row_div, ntok, nheads, qmap, box_rows, limit0, b_end, nt;
 };
+// Key tiles of an item: first the na tiles of the shared range [0, a_end) (the sink), then the tiles of the own
+// range from global key row b_start on.  The own range is fetched through the block tensor map at row
+// b_coord0 of that map, or, for the sink's own items, through the sink map (own_map = 1).
 struct WorkItem {
-    int kv_head, a_end, b_start, na, split;
+    int kv_head, a_end, b_start, na, split, b_coord0, own_map;
     QSlot s[2];
 };
 
@@ -137,6 +136,8 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             tail_rows = p.tail_rows_block; tail_heads = p.tail_heads_block; tail_tiles = p.tail_tiles_block;
             qmap_tail = 1;
             it.a_end = p.S;
+            it.b_coord0 = blk * p.B;
+            it.own_map = 0;
         } else {
             const int w2 = w - p.items_block;
             g = w2 / p.pairs_sink;
@@ -148,6 +149,8 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
             tail_rows = p.tail_rows_sink; tail_heads = p.tail_heads_sink; tail_tiles = p.tail_tiles_sink;
             qmap_tail = 2;
             it.a_end = 0;
+            it.b_coord0 = 0;
+            it.own_map = 1;
         }
         it.kv_head = g;
         it.b_start = seg_start;
@@ -197,6 +200,8 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int w, WorkItem
         const int split_lo = it.split * p.tiles_per_split * kTile;
         const int split_hi = split_lo + p.tiles_per_split * kTile;
         it.b_start = split_lo;
+        it.b_coord0 = split_lo;
+        it.own_map = 0;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
             const int qt = 2 * pi + x;
@@ -223,6 +228,7 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap tmap_q,
             const __grid_constant__ CUtensorMap tmap_q_tail_block, const __grid_constant__ CUtensorMap tmap_q_tail_sink,
+            const __grid_constant__ CUtensorMap tmap_k_sink, const __grid_constant__ CUtensorMap tmap_v_sink,
             const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
     using L = AttnSmem<D>;
     constexpr int NP = L::kPanels;
@@ -268,6 +274,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         tma_prefetch_desc(&tmap_q);
         tma_prefetch_desc(&tmap_q_tail_block);
         tma_prefetch_desc(&tmap_q_tail_sink);
+        tma_prefetch_desc(&tmap_k_sink);
+        tma_prefetch_desc(&tmap_v_sink);
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
     }
@@ -284,7 +292,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         if (atomicCAS(&p.hdr->status, 0, PEVLM_ETIMEOUT) == 0) p.hdr->detail = which * 1000000 + blockIdx.x;
     };
     auto wait = [&](uint32_t bar, uint32_t parity, int which) {
-        if (!mbar_wait(bar, parity, &abort_flag)) give_up(which);
+        if (!mbar_wait(bar, parity, &abort_flag, p.wait_limit_ns)) give_up(which);
     };
     // consumer side of the item queue: k-th item of this CTA, -1 = no more work
     auto next_item = [&](int k, WorkItem& it) {
@@ -329,7 +337,10 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     ++q_loads[x];
                 }
                 for (int j = 0; j < nt_max; ++j) {
-                    const int j0 = j < it.na ? j * kTile : it.b_start + (j - it.na) * kTile;
+                    // Rows past the end of the sink, and past the end of the block range, are outside their
+                    // tensor map and arrive as zeros: a ragged last tile never brings in a neighbour's rows.
+                    const bool shared_range = j < it.na || it.own_map != 0;
+                    const int j0 = j < it.na ? j * kTile : it.b_coord0 + (j - it.na) * kTile;
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const int slot = ring_idx % kRing, use = ring_idx / kRing;
@@ -337,7 +348,8 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                         mbar_arrive_expect_tx(bar_full + 8 * slot, L::kTileBytes);
                         for (int h = 0; h < NP; ++h)
                             tma_load_3d(smem_base + L::kRing0 + slot * L::kTileBytes + h * L::kPanelBytes,
-                                        kv ? &tmap_v : &tmap_k, h * 64, it.kv_head, j0, bar_full + 8 * slot);
+                                        shared_range ? (kv ? &tmap_v_sink : &tmap_k_sink) : (kv ? &tmap_v : &tmap_k),
+                                        h * 64, it.kv_head, j0, bar_full + 8 * slot);
                         ++ring_idx;
                     }
                 }
@@ -350,9 +362,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         int ring_base = 0;        // ring position of this item's K(0)
         int cnt[2] = {0, 0};      // tiles per slot before this item (phase of s_full / po)
         int q_uses[2] = {0, 0};   // items in which the slot was active so far
-#ifdef PEVLM_PROFILE
-        unsigned prof_po = 0, prof_full = 0, prof_t0 = static_cast<unsigned>(clock64()), prof_a = 0;
-#endif
         for (int k = 0;; ++k) {
             // every lane reads the item, one lane releases the queue slot
             wait(bar_item_full + 8 * (k & 1), (k >> 1) & 1, kWaitItem);
@@ -375,13 +384,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             auto ring_addr = [&](int idx) { return smem_base + L::kRing0 + ((ring_base + idx) % kRing) * L::kTileBytes; };
             auto wait_full = [&](int idx) {
                 const int g = ring_base + idx;
-#ifdef PEVLM_PROFILE
-                prof_a = static_cast<unsigned>(clock64());
-#endif
                 wait(bar_full + 8 * (g % kRing), (g / kRing) & 1, kWaitFull);
-#ifdef PEVLM_PROFILE
-                prof_full += static_cast<unsigned>(clock64()) - prof_a;
-#endif
             };
             auto commit_empty = [&](int idx) { mma_commit_elect(bar_empty + 8 * ((ring_base + idx) % kRing)); };
             // S_x = Q_x K(j)^T
@@ -397,13 +400,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             };
             // O_x += P_x V(j)
             auto issue_pv = [&](int x, int j) {
-#ifdef PEVLM_PROFILE
-                prof_a = static_cast<unsigned>(clock64());
-#endif
                 wait((kPvSplit > 0 ? bar_po_a : bar_po) + 8 * x, (cnt[x] + j) & 1, kWaitPO);
-#ifdef PEVLM_PROFILE
-                prof_po += static_cast<unsigned>(clock64()) - prof_a;
-#endif
                 PEVLM_STAMP(6, j, lane == 0 && x == 0);
                 // the previous item's output must have left TMEM before O is overwritten
                 if (j == 0 && q_uses[x] > 0) wait(bar_o_free + 8 * x, (q_uses[x] - 1) & 1, kWaitOFree);
@@ -487,13 +484,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 if (nt[x] > 0) ++q_uses[x];
             }
         }
-#ifdef PEVLM_PROFILE
-        if (lane == 0 && blockIdx.x == 0) {
-            p.hdr->pad[0] = static_cast<int32_t>((static_cast<unsigned>(clock64()) - prof_t0) >> 4);
-            p.hdr->pad[1] = static_cast<int32_t>(prof_po >> 4);
-            p.hdr->pad[2] = static_cast<int32_t>(prof_full >> 4);
-        }
-#endif
       }
     } else {
         // ------------------------------------------------------------- softmax and epilogue of slot x
@@ -507,10 +497,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
         int cnt = 0;        // tiles of this slot processed so far (phase of s_full)
         int uses = 0;       // items in which this slot was active so far
         int ring_base = 0;  // ring position of this item's K(0)
-#ifdef PEVLM_PROFILE
-        unsigned prof_busy = 0, prof_wait = 0, prof_t1 = 0, prof_t2 = static_cast<unsigned>(clock64()), prof_tiles = 0;
-        unsigned prof_ld = 0, prof_exp = 0;
-#endif
         for (int k = 0;; ++k) {
             WorkItem it;
             const int w = next_item(k, it);
@@ -549,10 +535,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                 const int nvalid = min(kTile, (j < na ? a_end : b_end) - j0);
                 const bool need_mask = (nvalid < kTile) || (j0 + kTile - 1 > limit0);
                 wait(my_s_full, cnt & 1, kWaitS);
-#ifdef PEVLM_PROFILE
-                prof_t1 = static_cast<unsigned>(clock64());
-                prof_wait += prof_t1 - prof_t2;
-#endif
                 PEVLM_STAMP(0 + x, j, (tid & 127) == 0);
                 PEVLM_STAMP_ITEM(3, k, tid == 0 && j == 0);
                 tc_fence_after_sync();
@@ -561,10 +543,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32 * c]));
                 tmem_wait_ld();
-#ifdef PEVLM_PROFILE
-                const unsigned prof_t_ld = static_cast<unsigned>(clock64());
-                prof_ld += prof_t_ld - prof_t1;
-#endif
                 if (need_mask) {
                     const int max_col = min(nvalid, my_limit - j0 + 1);
 #pragma unroll
@@ -635,20 +613,11 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
                     unpack_f32x2(add_f32x2(sm2[2], sm2[3]), b0, b1);
                     sum = (a0 + a1) + (b0 + b1);
                 }
-#ifdef PEVLM_PROFILE
-                const unsigned prof_t_exp = static_cast<unsigned>(clock64());
-                prof_exp += prof_t_exp - prof_t_ld;
-#endif
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(my_po);
                 PEVLM_STAMP(2 + x, j, (tid & 127) == 0);
                 PEVLM_STAMP_ITEM(4, k, tid == 0 && j == nt - 1);
-#ifdef PEVLM_PROFILE
-                prof_t2 = static_cast<unsigned>(clock64());
-                prof_busy += prof_t2 - prof_t1;
-                ++prof_tiles;
-#endif
                 l_run = l_run * alpha + sum;
             }
             // Epilogue, by the same thread (its registers are free now and it would only wait for the next
@@ -699,15 +668,6 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
             PEVLM_STAMP_ITEM(7, k, tid == 0);
             ++uses;
         }
-#ifdef PEVLM_PROFILE
-        if ((tid & 127) == 0 && blockIdx.x == 0) {
-            p.hdr->pad[8 + 8 * x] = static_cast<int32_t>(prof_busy >> 4);
-            p.hdr->pad[9 + 8 * x] = static_cast<int32_t>(prof_wait >> 4);
-            p.hdr->pad[10 + 8 * x] = static_cast<int32_t>(prof_tiles);
-            p.hdr->pad[11 + 8 * x] = static_cast<int32_t>(prof_ld >> 4);
-            p.hdr->pad[12 + 8 * x] = static_cast<int32_t>(prof_exp >> 4);
-        }
-#endif
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -717,8 +677,7 @@ attn_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtens
     }
 }
 
-cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tq_tail_block,
-                        const CUtensorMap& tq_tail_sink, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t stream) {
+cudaError_t launch_attn(const AttnParams& p, int head_dim, const AttnMaps& m, cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
     const size_t smem = attn_smem_bytes(head_dim);
     int dev = 0, sms = 0;
@@ -730,11 +689,11 @@ cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<128><<<grid, kAttnThreads, smem, stream>>>(p, tq, tq_tail_block, tq_tail_sink, tk, tv);
+        attn_kernel<128><<<grid, kAttnThreads, smem, stream>>>(p, m.q, m.q_tail_block, m.q_tail_sink, m.k_sink, m.v_sink, m.k, m.v);
     } else {
         e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attn_kernel<64><<<grid, kAttnThreads, smem, stream>>>(p, tq, tq_tail_block, tq_tail_sink, tk, tv);
+        attn_kernel<64><<<grid, kAttnThreads, smem, stream>>>(p, m.q, m.q_tail_block, m.q_tail_sink, m.k_sink, m.v_sink, m.k, m.v);
     }
     return cudaGetLastError();
 }

@@ -47,6 +47,7 @@ struct AttnParams {
     int32_t q_tiles;        // mode 1: ceil(Q / tok_per_tile)
     int32_t n_splits;       // mode 1
     int32_t tiles_per_split;// mode 1
+    uint64_t wait_limit_ns; // longest a single device-side wait may last before the launch reports PEVLM_ETIMEOUT
     float scale;            // softmax scale
     float scale_log2;       // scale * log2(e)
     __nv_bfloat16* o;       // mode 0: [n_video, Hq, d]
@@ -90,8 +91,19 @@ struct CopySegments {
 
 cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream);
 cudaError_t launch_copy_segments(const CopySegments& s, cudaStream_t stream);
-cudaError_t launch_attn(const AttnParams& p, int head_dim, const CUtensorMap& tq, const CUtensorMap& tq_tail_block,
-                        const CUtensorMap& tq_tail_sink, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t stream);
+// Tensor maps of one attention launch.  q: [rows, Hq, d] with a 128-token box; q_tail_*: the same tensor with the
+// box of a packed ragged tail (heads x tail rows).  K and V each have two maps so that a ragged last key tile
+// reads zeros past the end of its range instead of a neighbour's rows: *_sink covers cache rows [0, S), k / v
+// cover the context blocks of the call (base at the first block's row) or, for the question attention, the cache.
+struct AttnMaps {
+    CUtensorMap q, q_tail_block, q_tail_sink, k_sink, v_sink, k, v;
+};
+cudaError_t launch_attn(const AttnParams& p, int head_dim, const AttnMaps& m, cudaStream_t stream);
+cudaError_t launch_wait_selftest(WorkspaceHeader* hdr, uint64_t limit_ns, cudaStream_t stream);
+// device address of the built-in scratch array of pevlm_query_attn_noalloc on the current device
+int noalloc_scratch_for_current_device(void** out);
+int check_query_args(const pevlm_shape_t* s, const void* q_question, const void* k_cache, const void* v_cache,
+                     const void* o, const float* lse);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 size_t attn_smem_bytes(int head_dim);
 // error reporting shared by the host-side translation units: both record a text that

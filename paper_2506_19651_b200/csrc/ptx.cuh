@@ -48,11 +48,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` lives in shared memory: once any thread of the CTA has given
 // up on a wait, every later wait in the CTA gives up after a short grace period, so the
 // kernel always runs to its normal end (control flow is never altered by a timeout).
-// Returns false if the wait expired.
-constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;  // 0.4 s: orders of magnitude above any legitimate wait
+// `limit_ns` is the longest a single wait may last (a launch parameter: the library's calls pass
+// kDefaultWaitLimitNs, orders of magnitude above any legitimate wait).  Returns false if the wait expired.
+constexpr uint64_t kDefaultWaitLimitNs = 400ull * 1000 * 1000;  // 0.4 s
 constexpr uint64_t kAbortGraceNs = 20ull * 1000;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
@@ -60,7 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             const uint64_t dt = globaltimer_ns() - t0;
-            const uint64_t lim = (*abort_flag) ? kAbortGraceNs : kWaitLimitNs;
+            const uint64_t lim = (*abort_flag) ? kAbortGraceNs : limit_ns;
             if (dt > lim) {
                 *abort_flag = 1;
                 return false;

@@ -24,8 +24,10 @@ static __device__ __align__(256) unsigned char g_query_scratch[kScratchBytes];
 std::mutex g_setup_mutex;
 void* g_scratch_ptr[kMaxDevices] = {};
 
+}  // namespace
+
 // Once per device, with that device current: resolve the device address of the scratch array.
-int scratch_for_current_device(void** out) {
+int pevlm::noalloc_scratch_for_current_device(void** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return pevlm::cuda_fail(e, "cudaGetDevice");
@@ -41,10 +43,12 @@ int scratch_for_current_device(void** out) {
     return PEVLM_OK;
 }
 
-}  // namespace
-
 extern "C" int pevlm_query_attn_noalloc(const pevlm_shape_t* shape, const void* q_question, const void* k_cache,
                                         const void* v_cache, void* o, float* lse, void* stream) {
+    // Everything that can be refused on the host is refused before the device is touched: a bad shape or
+    // pointer by the same checks as the workspace entry point, then a shape beyond the array.
+    const int bad = pevlm::check_query_args(shape, q_question, k_cache, v_cache, o, lse);
+    if (bad != PEVLM_OK) return bad;
     const size_t need = pevlm_workspace_bytes(shape, PEVLM_WS_QUERY);
     if (need > kScratchBytes) {
         char text[160];
@@ -53,7 +57,7 @@ extern "C" int pevlm_query_attn_noalloc(const pevlm_shape_t* shape, const void* 
         return pevlm::fail_with_text(PEVLM_EWORKSPACE, text);
     }
     void* scratch = nullptr;
-    const int rc = scratch_for_current_device(&scratch);
+    const int rc = pevlm::noalloc_scratch_for_current_device(&scratch);
     if (rc != PEVLM_OK) return rc;
     // Same kernels as pevlm_query_attn, with the built-in array as the workspace.  The status
     // header at its start is cleared on the stream by that call; the partials are fully

@@ -130,13 +130,13 @@ def make_qkv(w: Workload, layer: int = 0):
 
 
 def sample_rows(w: Workload, n_random: int, seed: int = 7, tile: int = 128) -> np.ndarray:
-    """A stratified sample of token rows: segment, block and tile edges, the whole
-    question block, plus seeded random rows.  Sorted, unique, all < L."""
+    """A stratified sample of token rows: the first and last two rows and every tile edge (edge - 1, edge,
+    edge + 1) of the sink and of EVERY context block, the whole question block, plus seeded random rows.
+    Sorted, unique, all < L."""
     rows = set()
     nv = w.n_video
     segs = [(0, w.S)] + [(w.S + b * w.B, w.S + (b + 1) * w.B) for b in range(w.N)]
-    pick_blocks = sorted(set([0, 1, 2, w.N // 2, w.N - 1, w.N]) & set(range(len(segs))))
-    for si in pick_blocks:
+    for si in range(len(segs)):
         a, e = segs[si]
         if e <= a:
             continue

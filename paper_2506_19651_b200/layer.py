@@ -12,23 +12,28 @@ from . import binding as pb
 class LayerBuffers:
     """Device buffers of one layer pass, allocated once and reused across steps."""
 
-    def __init__(self, shape: pb.Shape, device="cuda"):
+    def __init__(self, shape: pb.Shape, device="cuda", alloc=None):
+        """`alloc(shape, dtype, zero)` replaces torch.empty / torch.zeros (the tests pass an allocator that puts
+        guard bytes around every buffer)."""
         import torch
         s = shape
         nv, Q, L = s.n_video, s.query_len, s.L
         Hq, Hkv, d = s.num_q_heads, s.num_kv_heads, s.head_dim
         bf, f32 = torch.bfloat16, torch.float32
+        if alloc is None:
+            def alloc(shp, dtype, zero=False):
+                return (torch.zeros if zero else torch.empty)(shp, dtype=dtype, device=device)
         self.shape = s
-        self.q_video = torch.empty((max(nv, 1), Hq, d), dtype=bf, device=device)   # roped in place
-        self.q_question = torch.empty((max(Q, 1), Hq, d), dtype=bf, device=device)
-        self.k_cache = torch.empty((L, Hkv, d), dtype=bf, device=device)
-        self.v_cache = torch.empty((L, Hkv, d), dtype=bf, device=device)
-        self.o_video = torch.empty((max(nv, 1), Hq, d), dtype=bf, device=device)
-        self.lse_video = torch.empty((Hq, max(nv, 1)), dtype=f32, device=device)
-        self.o_question = torch.empty((max(Q, 1), Hq, d), dtype=bf, device=device)
-        self.lse_question = torch.empty((Hq, max(Q, 1)), dtype=f32, device=device)
-        self.ws_prefill = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_PREFILL), dtype=torch.uint8, device=device)
-        self.ws_query = torch.zeros(pb.pevlm_workspace_bytes(s, pb.WS_QUERY), dtype=torch.uint8, device=device)
+        self.q_video = alloc((max(nv, 1), Hq, d), bf)   # roped copy of the video queries
+        self.q_question = alloc((max(Q, 1), Hq, d), bf)
+        self.k_cache = alloc((L, Hkv, d), bf)
+        self.v_cache = alloc((L, Hkv, d), bf)
+        self.o_video = alloc((max(nv, 1), Hq, d), bf)
+        self.lse_video = alloc((Hq, max(nv, 1)), f32)
+        self.o_question = alloc((max(Q, 1), Hq, d), bf)
+        self.lse_question = alloc((Hq, max(Q, 1)), f32)
+        self.ws_prefill = alloc((pb.pevlm_workspace_bytes(s, pb.WS_PREFILL),), torch.uint8, zero=True)
+        self.ws_query = alloc((pb.pevlm_workspace_bytes(s, pb.WS_QUERY),), torch.uint8, zero=True)
 
 
 KERNELS_PER_PASS = 7  # rope, V copy, prefill attention, rope, V copy, question attention, merge
@@ -62,7 +67,7 @@ def layer_forward(buf: LayerBuffers, q, k, v, mark=None):
     return buf
 
 
-def ragged_layer_forward(q, k, v, S, B, N, B_last, Q, theta, scale=0.0):
+def ragged_layer_forward(q, k, v, S, B, N, B_last, Q, theta, scale=0.0, alloc=None):
     """Layer pass over a video whose length is not a multiple of the block length: N context blocks, the
     first N-1 of B tokens, the last one of B_last < B tokens (the uniform partition of Sec. 3.2.1 with the
     remainder as one shorter block).  q [L,Hq,d], k, v [L,Hkv,d] un-roped device tensors of the whole
@@ -70,6 +75,7 @@ def ragged_layer_forward(q, k, v, S, B, N, B_last, Q, theta, scale=0.0):
 
     The uniform prefix runs through pevlm_parallel_prefill_attn, the last block through pevlm_block_attn
     against the same cache, the question through pevlm_query_attn; positions are the global ones.
+    `alloc(shape, dtype, zero)` replaces torch.empty / torch.zeros (see LayerBuffers).
     """
     import torch
     Hq, Hkv, d = q.shape[1], k.shape[1], q.shape[2]
@@ -81,19 +87,22 @@ def ragged_layer_forward(q, k, v, S, B, N, B_last, Q, theta, scale=0.0):
     s_all = pb.make_shape(nv, 1, 0, Q, Hq, Hkv, d, theta=theta, scale=scale)          # [video | question]
     s_full = pb.make_shape(S, B, N - 1, 0, Hq, Hkv, d, theta=theta, scale=scale)      # uniform prefix
     s_last = pb.make_shape(S, B_last, 1, 0, Hq, Hkv, d, theta=theta, scale=scale)     # the shorter last block
-    q_roped = torch.empty((L, Hq, d), dtype=bf, device=dev)
-    k_cache = torch.empty((L, Hkv, d), dtype=bf, device=dev)
-    v_cache = torch.empty((L, Hkv, d), dtype=bf, device=dev)
-    o_video = torch.empty((nv, Hq, d), dtype=bf, device=dev)
-    lse_video = torch.empty((Hq, nv), dtype=f32, device=dev)
-    lse_last = torch.empty((Hq, B_last), dtype=f32, device=dev)
-    o_question = torch.empty((max(Q, 1), Hq, d), dtype=bf, device=dev)
-    lse_question = torch.empty((Hq, max(Q, 1)), dtype=f32, device=dev)
-    ws = [torch.zeros(pb.pevlm_workspace_bytes(s, which), dtype=torch.uint8, device=dev)
+    if alloc is None:
+        def alloc(shp, dtype, zero=False):
+            return (torch.zeros if zero else torch.empty)(shp, dtype=dtype, device=dev)
+    q_roped = alloc((L, Hq, d), bf)
+    k_cache = alloc((L, Hkv, d), bf)
+    v_cache = alloc((L, Hkv, d), bf)
+    o_video = alloc((nv, Hq, d), bf)
+    lse_video = alloc((Hq, nv), f32)
+    lse_last = alloc((Hq, B_last), f32)
+    o_question = alloc((max(Q, 1), Hq, d), bf)
+    lse_question = alloc((Hq, max(Q, 1)), f32)
+    ws = [alloc((pb.pevlm_workspace_bytes(s, which),), torch.uint8, zero=True)
           for s, which in ((s_full, pb.WS_PREFILL), (s_last, pb.WS_PREFILL), (s_all, pb.WS_QUERY))]
     pb.pevlm_rope_qk(s_all, q, k, q_roped, k_cache, 0, L)
     pb.pevlm_assemble_kv(s_all, None, v[:nv], None, v[nv:] if Q > 0 else None, k_cache, v_cache)
-    lse_full = torch.empty((Hq, max(nv_full, 1)), dtype=f32, device=dev)
+    lse_full = alloc((Hq, max(nv_full, 1)), f32)
     if nv_full > 0:
         pb.pevlm_parallel_prefill_attn(s_full, q_roped[:nv_full], k_cache[:nv_full], v_cache[:nv_full],
                                        o_video[:nv_full], lse_full, ws[0])

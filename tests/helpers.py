@@ -25,6 +25,32 @@ def bits_to_f64(b):
     return inputs.bf16_bits_to_f64(b)
 
 
+class GuardedAllocator:
+    """Device buffers with canary bytes before and after each one (the stand-in for a memory checker): every
+    buffer sits inside a larger allocation whose first and last 4 KiB (the tail guard starts at the buffer's
+    last byte + 1) hold a known pattern; check() asserts that no kernel wrote there."""
+    GUARD = 4096
+    PATTERN = 0xA5
+
+    def __init__(self):
+        self.items = []
+
+    def __call__(self, shape, dtype, zero=False):
+        import torch
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((2 * self.GUARD + (n + 255) // 256 * 256,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        view = raw[self.GUARD:self.GUARD + n].view(dtype).view(shape)
+        if zero:
+            view.zero_()
+        self.items.append((raw, n))
+        return view
+
+    def check(self):
+        for raw, n in self.items:
+            assert bool((raw[:self.GUARD] == self.PATTERN).all()), "write before the start of a buffer"
+            assert bool((raw[self.GUARD + n:] == self.PATTERN).all()), "write past the end of a buffer"
+
+
 def gpu_shape(w: inputs.Workload, full_causal=False, scale=0.0):
     from paper_2506_19651_b200 import binding as pb
     return pb.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d, theta=w.theta, scale=scale,
@@ -41,12 +67,14 @@ def run_gpu_layer(w: inputs.Workload, q, k, v, full_causal=False):
     from paper_2506_19651_b200 import binding as pb
     from paper_2506_19651_b200.layer import LayerBuffers, layer_forward
     s = gpu_shape(w, full_causal)
-    buf = LayerBuffers(s)
+    guard = GuardedAllocator()
+    buf = LayerBuffers(s, alloc=guard)
     layer_forward(buf, to_dev(q), to_dev(k), to_dev(v))
     torch.cuda.synchronize()
     for ws in (buf.ws_prefill, buf.ws_query):
         st, det = pb.pevlm_read_status(ws)
         assert st == 0, f"device wait expired: status {st} detail {det}"
+    guard.check()   # no store outside q_video, the caches, o, lse or the workspaces (partials included)
     nv = w.n_video
     return {
         "q_video": to_bits(buf.q_video[:nv]), "q_question": to_bits(buf.q_question[:w.Q]),

@@ -84,6 +84,14 @@ def test_argument_errors_before_launch(lib):
     f = lib.pevlm_parallel_prefill_attn
     assert f(C.byref(good), None, p16, p16, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
     assert f(C.byref(good), odd, p16, p16, p16, None, ws, 1 << 20, None) == pb.PEVLM_EALIGN
+    # the attention outputs are written with 32-byte vector stores: an `o` at 16 mod 32 is refused on the
+    # host (nothing is launched), for every call that writes one
+    o16 = C.c_void_p(4096 + 16)
+    assert f(C.byref(good), p16, p16, p16, o16, None, ws, 1 << 20, None) == pb.PEVLM_EALIGN
+    assert lib.pevlm_block_attn(C.byref(good), p16, p16, p16, 64, 64 + 512, o16, None, ws, 1 << 20, None) == pb.PEVLM_EALIGN
+    assert lib.pevlm_query_attn(C.byref(good), p16, p16, p16, o16, None, ws, 1 << 30, None) == pb.PEVLM_EALIGN
+    assert lib.pevlm_query_attn_noalloc(C.byref(good), p16, p16, p16, o16, None, None) == pb.PEVLM_EALIGN
+    assert f(C.byref(good), p16, p16, p16, p16, None, C.c_void_p(4096 + 128), 1 << 20, None) == pb.PEVLM_EALIGN
     assert f(C.byref(good), p16, p16, p16, p16, None, None, 1 << 20, None) == pb.PEVLM_EWORKSPACE
     assert f(C.byref(good), p16, p16, p16, p16, None, ws, 8, None) == pb.PEVLM_EWORKSPACE
     assert f(None, p16, p16, p16, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
@@ -96,6 +104,8 @@ def test_argument_errors_before_launch(lib):
         assert lib.pevlm_query_attn(C.byref(bad), p16, p16, p16, p16, None, ws, 1 << 30, None) == code, field
         assert lib.pevlm_rope_qk(C.byref(bad), p16, p16, p16, p16, 0, 8, None, None) == code, field
         assert lib.pevlm_assemble_kv(C.byref(bad), p16, p16, p16, p16, p16, p16, None) == code, field
+        # the no-workspace entry point names the same error, before it touches the device
+        assert lib.pevlm_query_attn_noalloc(C.byref(bad), p16, p16, p16, p16, None, None) == code, field
     assert lib.pevlm_rope_qk(C.byref(good), p16, None, None, None, 0, 8, None, None) == pb.PEVLM_EINVAL
     assert lib.pevlm_rope_qk(C.byref(good), odd, None, odd, None, 0, 8, None, None) == pb.PEVLM_EALIGN
     assert lib.pevlm_rope_qk(C.byref(good), p16, None, p16, None, -1, 8, None, None) == pb.PEVLM_EINVAL
@@ -115,6 +125,14 @@ def test_argument_errors_before_launch(lib):
     assert g(C.byref(good), p16, p16, p16, 64, 64 + nb, p16, None, None, 0, None) == pb.PEVLM_EWORKSPACE
     fc = pb.make_shape(64, 128, 4, 32, 4, 2, 64, mask_mode=pb.MASK_FULL_CAUSAL)
     assert g(C.byref(fc), p16, p16, p16, 64, 64 + nb, p16, None, ws, 1 << 20, None) == pb.PEVLM_EINVAL
+    assert lib.pevlm_query_attn_noalloc(C.byref(good), None, p16, p16, p16, None, None) == pb.PEVLM_EINVAL
+    # wait self-test: workspace, alignment and the range of the limit are checked on the host
+    t = lib.pevlm_selftest_wait_expiry
+    assert t(None, 256, 1000000, None) == pb.PEVLM_EWORKSPACE
+    assert t(ws, 16, 1000000, None) == pb.PEVLM_EWORKSPACE
+    assert t(C.c_void_p(1024 + 8), 256, 1000000, None) == pb.PEVLM_EALIGN
+    assert t(ws, 256, 10, None) == pb.PEVLM_EINVAL
+    assert t(ws, 256, 10 ** 10, None) == pb.PEVLM_EINVAL
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

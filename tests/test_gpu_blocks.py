@@ -31,9 +31,12 @@ def test_ragged_last_block(S, B, N, Q, B_last, Hq, Hkv, d):
     theta = 1e6
     w = inputs.Workload("t", S, B, N, Q, Hq, Hkv, d, theta, S > 0, 4321, B_last=B_last)
     q, k, v = inputs.make_qkv(w)
-    o_v, lse_v, o_q, lse_q, ws = ragged_layer_forward(to_dev(q), to_dev(k), to_dev(v), S, B, N, B_last, Q, theta)
+    from helpers import GuardedAllocator
+    guard = GuardedAllocator()
+    o_v, lse_v, o_q, lse_q, ws = ragged_layer_forward(to_dev(q), to_dev(k), to_dev(v), S, B, N, B_last, Q, theta, alloc=guard)
     torch.cuda.synchronize()
     _status_ok(*ws)
+    guard.check()   # canary bytes around every buffer of the pass, the block-range call's o and lse included
     nv = w.n_video
     qr, kr = oracle.rope(q, theta), oracle.rope(k, theta)
     sh = oracle.make_shape(S, B, N, Q, Hq, Hkv, d, B_last=B_last)
@@ -186,3 +189,39 @@ def test_sequences_of_different_shapes_share_one_cache_buffer():
         lse_gpu = np.concatenate([lse_v.double().cpu().numpy().T, lse_q.double().cpu().numpy().T])
         assert np.abs(o_gpu - o).max() <= O_TOL
         assert np.abs(lse_gpu - lse).max() <= LSE_TOL
+
+
+@pytest.mark.parametrize("S,B,N,Hq,Hkv,d", [(100, 75, 2, 4, 2, 128), (37, 130, 1, 14, 2, 128), (200, 333, 3, 8, 4, 64)])
+def test_block_range_ignores_the_rest_of_the_cache(S, B, N, Hq, Hkv, d):
+    """The cache outside the sink rows and the block range holds NaN bit patterns (an uninitialised slot of a
+    streaming window); S and B are not multiples of 16, so the ragged last key tiles end inside a 16-row MMA
+    step.  The outputs must be those of the oracle (a zero probability times a NaN value row would be NaN),
+    and nothing may be written outside o and lse (canary bytes around both)."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    from helpers import GuardedAllocator
+    theta = 1e6
+    w = inputs.Workload("t", S, B, N, 0, Hq, Hkv, d, theta, True, 555)
+    q, k, v = inputs.make_qkv(w)
+    qr, kr = oracle.rope(q, theta), oracle.rope(k, theta)
+    gap, tail = 53, 91                              # unused rows between the sink and the blocks, and after them
+    first = S + gap
+    rows = first + N * B + tail
+    nan = torch.full((rows, Hkv, d), -1, dtype=torch.int16, device="cuda").view(torch.bfloat16)   # 0xFFFF = NaN
+    kc, vc = nan.clone(), nan.clone()
+    kc[:S], vc[:S] = to_dev(kr[:S]), to_dev(v[:S])
+    kc[first:first + N * B], vc[first:first + N * B] = to_dev(kr[S:]), to_dev(v[S:])
+    s = pb.make_shape(S, B, N, 0, Hq, Hkv, d, theta=theta)
+    guard = GuardedAllocator()
+    o = guard((N * B, Hq, d), torch.bfloat16)
+    lse = guard((Hq, N * B), torch.float32)
+    ws = guard((pb.pevlm_workspace_bytes(s, pb.WS_PREFILL),), torch.uint8, zero=True)
+    pb.pevlm_block_attn(s, to_dev(qr[S:]), kc, vc, first, rows, o, lse, ws)
+    torch.cuda.synchronize()
+    _status_ok(ws)
+    guard.check()
+    o_ref, lse_ref = oracle.attn_rows(oracle.make_shape(S, B, N, 0, Hq, Hkv, d), qr, kr, v, np.arange(S, w.L, dtype=np.int64))
+    got = bits_to_f64(to_bits(o))
+    assert np.isfinite(got).all()
+    assert np.abs(got - o_ref).max() <= O_TOL
+    assert np.abs(lse.double().cpu().numpy().T - lse_ref).max() <= LSE_TOL

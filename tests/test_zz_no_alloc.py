@@ -32,6 +32,7 @@ def _case(S, B, N, Q, Hq, Hkv, d, seed):
     pb.pevlm_query_attn_noalloc(s, dq, dk, dv, o_new, lse_new)
     torch.cuda.synchronize()
     assert pb.pevlm_read_status(ws)[0] == 0
+    assert pb.pevlm_read_status(None) == (0, 0)      # the status header of the built-in array
     a, b = bits_to_f64(to_bits(o_new)), bits_to_f64(to_bits(o_ref))
     assert np.abs(a - b).max() <= O_TOL
     assert (lse_new - lse_ref).abs().max().item() <= LSE_TOL

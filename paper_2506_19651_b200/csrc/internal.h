@@ -75,7 +75,7 @@ struct RopeParams {
     int64_t first_token;
     int64_t n_tokens;
     int32_t Hq, Hkv;  // heads to process of each tensor (0 = skip tensor)
-    int32_t head_split;  // thread groups sharing one token's heads (set by launch_rope)
+    int32_t head_split;  // slots sharing one token's heads (set by launch_rope)
     // multimodal RoPE: pos3 != NULL selects it; rotary pair i takes its position from component 0 for
     // i < sec_end0, component 1 for i < sec_end1, else component 2; pos3 is [3, n_tokens]
     const int32_t* pos3;

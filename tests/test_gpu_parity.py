@@ -39,6 +39,28 @@ def test_rope_bit_exact(n, Hq, Hkv, d, theta, first):
     np.testing.assert_array_equal(to_bits(qd), q)  # untouched
 
 
+def test_rope_bit_exact_on_edge_values():
+    """Zeros of both signs, the smallest and largest finite bf16 values and subnormals in every position of a
+    rotation pair: the kernel widens bf16 to fp64 with integer arithmetic on the common path and must still
+    agree with the oracle bit for bit."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    special = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x007F, 0x0080, 0x8080, 0x7F7F, 0xFF7F, 0x3F80, 0xBF80,
+                        0x0100, 0x3F81, 0x4049, 0x00FF, 0x7F00], dtype=np.uint16)
+    n, Hq, Hkv, d = 64, 4, 2, 128
+    rng = np.random.default_rng(11)
+    q = special[rng.integers(0, special.size, size=(n, Hq, d))]
+    k = special[rng.integers(0, special.size, size=(n, Hkv, d))]
+    w = wl(n, 1, 0, 0, Hq, Hkv, d, 1e6)
+    s = gpu_shape(w)
+    qd, kd = to_dev(q), to_dev(k)
+    qo, ko = torch.empty_like(qd), torch.empty_like(kd)
+    pb.pevlm_rope_qk(s, qd, kd, qo, ko, 12345, n)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_bits(qo), oracle.rope(q, 1e6, first_pos=12345))
+    np.testing.assert_array_equal(to_bits(ko), oracle.rope(k, 1e6, first_pos=12345))
+
+
 # ---------------------------------------------------------------- KV assembly (Eq. 5 key set)
 
 def test_assemble_kv_bit_exact():

@@ -8,11 +8,7 @@ namespace pevlm {
 
 constexpr int kRopeThreads = 256;
 
-#ifndef PEVLM_ROPE_PREFETCH
-#define PEVLM_ROPE_PREFETCH 2
-#endif
-constexpr int kPrefetch = PEVLM_ROPE_PREFETCH;   // heads whose loads are in flight while one head is rotated
-constexpr int kRopeCtasPerSm = 4;                // resident CTAs per SM the register budget is set for
+constexpr int kRopeCtasPerSm = 4;  // resident CTAs per SM of the long-range form (its register budget: 64)
 
 // 16-byte accesses that do not allocate in L1 (every byte is touched once)
 __device__ __forceinline__ uint4 ld_stream(const __nv_bfloat16* p) {
@@ -45,18 +41,25 @@ __device__ __forceinline__ uint32_t f64x2_to_bf16x2_bits(double lo, double hi) {
 // these groups.  The kernel is bound by the bytes it keeps in flight (resident warps x outstanding loads) and
 // registers bound the resident warps, so the (cos, sin) pairs sit in a thread-private column of shared memory
 // rather than in 32 registers (4 resident CTAs per SM instead of 3) and the loads of the next two heads are
-// issued before a head is rotated.  No block-level synchronisation.  The heads of a token can be split over
+// issued before a head is rotated (template flag LONG).  Short ranges (the question block, a streamed block)
+// take the other form, which keeps the pairs in registers, uses no shared memory and fetches one head at a time:
+// a launch that uses shared memory made the attention launch that follows two launches later start about 9 us
+// later (the SMs change their shared-memory configuration), which a short range cannot pay back.
+// No block-level synchronisation.  The heads of a token can be split over
 // `head_split` slots, each evaluating the token's angles itself, for short token ranges (the question block),
 // so that the launch still fills the machine.
 // MODE 0: one position per token.  MODE 1, 2: the multimodal form, where a rotary pair's section picks the
 // position component; 1 when the section boundaries are multiples of 8 pairs (16/24/24 at d = 128), so that a
 // thread's 8 pairs share one component, 2 in general (a component per pair).
-template <int D, int MODE>
-__global__ void __launch_bounds__(kRopeThreads, kRopeCtasPerSm) rope_kernel(const __grid_constant__ RopeParams p) {
+template <int D, int MODE, bool LONG>
+__global__ void __launch_bounds__(kRopeThreads, LONG ? kRopeCtasPerSm : 1) rope_kernel(const __grid_constant__ RopeParams p) {
+    constexpr int kPrefetch = LONG ? 2 : 0;  // heads whose loads are in flight while one head is rotated
     constexpr int HALF = D / 2;
     constexpr int TPT = HALF / 8;                  // threads per slot
     constexpr int SLOTS_PER_CTA = kRopeThreads / TPT;
-    __shared__ double2 cs_sn[8][kRopeThreads];     // [pair of the thread][thread]: conflict-free 16-byte accesses
+    // [pair of the thread][thread]: conflict-free 16-byte accesses (one dummy element in the short form)
+    __shared__ double2 cs_sn[LONG ? 8 : 1][LONG ? kRopeThreads : 1];
+    double cs[LONG ? 1 : 8], sn[LONG ? 1 : 8];
     const int v = threadIdx.x % TPT;
     const int i0 = v * 8;
     const int heads = p.Hq + p.Hkv;
@@ -86,7 +89,12 @@ __global__ void __launch_bounds__(kRopeThreads, kRopeCtasPerSm) rope_kernel(cons
             const double ang = __dmul_rn(static_cast<double>(pe), p.inv_freq[i0 + e]);
             double sv, cv;
             sincos(ang, &sv, &cv);
-            cs_sn[e][threadIdx.x] = make_double2(cv, sv);
+            if (LONG) {
+                cs_sn[e][threadIdx.x] = make_double2(cv, sv);
+            } else {
+                cs[e] = cv;
+                sn[e] = sv;
+            }
         }
         auto addr_of = [&](int h, const __nv_bfloat16*& src, __nv_bfloat16*& dst) {
             if (h < p.Hq) {
@@ -136,8 +144,15 @@ __global__ void __launch_bounds__(kRopeThreads, kRopeCtasPerSm) rope_kernel(cons
                 for (int e = 0; e < 2; ++e) {
                     const double a = bf16_bits_to_f64((lo_w[w] >> (16 * e)) & 0xFFFFu);
                     const double b = bf16_bits_to_f64((hi_w[w] >> (16 * e)) & 0xFFFFu);
-                    const double2 t = cs_sn[2 * w + e][threadIdx.x];
-                    const double c = t.x, s = t.y;
+                    double c, s;
+                    if (LONG) {
+                        const double2 t = cs_sn[2 * w + e][threadIdx.x];
+                        c = t.x;
+                        s = t.y;
+                    } else {
+                        c = cs[2 * w + e];
+                        s = sn[2 * w + e];
+                    }
                     ra[e] = __dsub_rn(__dmul_rn(a, c), __dmul_rn(b, s));
                     rb[e] = __dadd_rn(__dmul_rn(b, c), __dmul_rn(a, s));
                 }
@@ -163,15 +178,22 @@ cudaError_t launch_rope(const RopeParams& p, int head_dim, cudaStream_t stream) 
     const int64_t cap = 2 * resident;  // CTAs stride over the remaining groups
     const unsigned grid = static_cast<unsigned>(groups < cap ? groups : cap);
     const int mode = !q.pos3 ? 0 : ((q.sec_end0 | q.sec_end1) & 7) == 0 ? 1 : 2;
+    const bool long_range = q.head_split == 1 && groups >= resident;  // at least one full round of resident CTAs
+#define PEVLM_ROPE_LAUNCH(D_, M_)                                                                   \
+    do {                                                                                            \
+        if (long_range) rope_kernel<D_, M_, true><<<grid, kRopeThreads, 0, stream>>>(q);            \
+        else rope_kernel<D_, M_, false><<<grid, kRopeThreads, 0, stream>>>(q);                      \
+    } while (0)
     if (head_dim == 128) {
-        if (mode == 0) rope_kernel<128, 0><<<grid, kRopeThreads, 0, stream>>>(q);
-        else if (mode == 1) rope_kernel<128, 1><<<grid, kRopeThreads, 0, stream>>>(q);
-        else rope_kernel<128, 2><<<grid, kRopeThreads, 0, stream>>>(q);
+        if (mode == 0) PEVLM_ROPE_LAUNCH(128, 0);
+        else if (mode == 1) PEVLM_ROPE_LAUNCH(128, 1);
+        else PEVLM_ROPE_LAUNCH(128, 2);
     } else {
-        if (mode == 0) rope_kernel<64, 0><<<grid, kRopeThreads, 0, stream>>>(q);
-        else if (mode == 1) rope_kernel<64, 1><<<grid, kRopeThreads, 0, stream>>>(q);
-        else rope_kernel<64, 2><<<grid, kRopeThreads, 0, stream>>>(q);
+        if (mode == 0) PEVLM_ROPE_LAUNCH(64, 0);
+        else if (mode == 1) PEVLM_ROPE_LAUNCH(64, 1);
+        else PEVLM_ROPE_LAUNCH(64, 2);
     }
+#undef PEVLM_ROPE_LAUNCH
     return cudaGetLastError();
 }
 

@@ -444,7 +444,6 @@ int pevlm_query_attn(const pevlm_shape_t* s, const void* q_question, const void*
         if (e != cudaSuccess) return cuda_fail(e, "question attention launch");
         MergeParams m;
         m.Q = p.Q; m.Hq = p.Hq; m.d = d; m.n_splits = p.n_splits;
-        m.striped_row0 = static_cast<int64_t>(p.Q) * p.Hq;
         m.part_o = p.part_o; m.part_lse = p.part_lse;
         m.o = static_cast<__nv_bfloat16*>(o) + qoff;
         m.lse = lse ? lse + static_cast<int64_t>(b) * p.Hq * p.Q : nullptr;

@@ -59,7 +59,6 @@ struct AttnParams {
 
 struct MergeParams {
     int32_t Q, Hq, d, n_splits;
-    int64_t striped_row0;  // rows (token * Hq + head) from here on have 2 * n_splits partials (Q * Hq = none)
     const float* part_o;
     const float* part_lse;
     __nv_bfloat16* o;  // [Q, Hq, d]

@@ -9,7 +9,7 @@ namespace pevlm {
 
 constexpr int kMergeThreads = 256;
 constexpr int kMergeChunk = 16;      // partial rows whose loads are in flight together
-constexpr int kMergeMaxParts = 320;  // >= 2 * the largest split count (one split per SM at most)
+constexpr int kMergeMaxParts = 160;  // >= the largest split count (one split per SM at most)
 
 // Many rows (a prefill-sized question block): one thread per (row, 4 output columns), the splits one after
 // another; tens of thousands of threads hide the latency of the dependent loads.
@@ -20,7 +20,7 @@ __global__ void merge_kernel(const __grid_constant__ MergeParams p) {
     if (idx >= rows * vec_per_row) return;
     const int64_t row = idx / vec_per_row;  // = tok * Hq + head
     const int v = static_cast<int>(idx % vec_per_row);
-    const int n = row >= p.striped_row0 ? 2 * p.n_splits : p.n_splits;
+    const int n = p.n_splits;
     float m = -INFINITY;
     for (int s = 0; s < n; ++s) m = fmaxf(m, p.part_lse[s * rows + row]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -51,8 +51,7 @@ __global__ void merge_kernel(const __grid_constant__ MergeParams p) {
 // everything that can be fetched side by side is: the first chunk of partial rows and all of the row's lse_s
 // (lane l takes splits l, l + 32, ...) are requested together; the lanes reduce the maximum and the sum, leave
 // the normalised weights in shared memory, and the partial rows follow in chunks of kMergeChunk, all loads of a
-// chunk issued before the first is used.  Rows whose query tile ran striped over the two slots of a CTA
-// (row >= striped_row0) have two banks of partials, n_splits each; the other rows only the first bank.
+// chunk issued before the first is used.
 __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(const __grid_constant__ MergeParams p) {
     __shared__ float weights[kMergeThreads / 32][kMergeMaxParts];
     const int lane = threadIdx.x & 31;
@@ -60,7 +59,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(const __grid_
     const int64_t row = static_cast<int64_t>(blockIdx.x) * (kMergeThreads / 32) + (threadIdx.x >> 5);
     const int64_t rows = static_cast<int64_t>(p.Q) * p.Hq;
     if (row >= rows) return;
-    const int n = row >= p.striped_row0 ? 2 * p.n_splits : p.n_splits;
+    const int n = p.n_splits;
     const bool col_ok = lane * 4 < p.d;
     auto load_chunk = [&](int s0, float4 (&o)[kMergeChunk]) {
 #pragma unroll
@@ -117,7 +116,7 @@ cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream) {
     const int64_t rows = static_cast<int64_t>(p.Q) * p.Hq;
     if (rows <= 0) return cudaSuccess;
     const int rows_per_cta = kMergeThreads / 32;
-    if (rows <= static_cast<int64_t>(kNumSms) * rows_per_cta && 2 * p.n_splits <= kMergeMaxParts) {
+    if (rows <= static_cast<int64_t>(kNumSms) * rows_per_cta && p.n_splits <= kMergeMaxParts) {
         // at most one CTA per SM of warp-per-row work: the latency-oriented form
         merge_rows_kernel<<<static_cast<unsigned>((rows + rows_per_cta - 1) / rows_per_cta), kMergeThreads, 0, stream>>>(p);
     } else {

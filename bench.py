@@ -79,6 +79,10 @@ def oracle_sample(w, q, k, v, target_seconds, seed=3):
     with the measured time, the rows and pairs covered and the implied whole-layer figures."""
     from oracle import api as oracle
     sh = oracle.make_shape(w.S, w.B, w.N, w.Q, w.Hq, w.Hkv, w.d)
+    if "TORCHELASTIC_RUN_ID" in os.environ and oracle.num_threads() == 1:
+        # the launcher pins OMP_NUM_THREADS to 1 for its ranks; the oracle runs on rank 0 alone and takes the
+        # cores this process may use, as it does when started without a launcher
+        oracle.set_num_threads(len(os.sched_getaffinity(0)))
     cores = oracle.num_threads()
     t0 = time.perf_counter()
     qr = oracle.rope(q, w.theta)

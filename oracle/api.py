@@ -61,6 +61,10 @@ def num_threads() -> int:
     return int(lib().oracle_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    lib().oracle_set_num_threads(C.c_int(int(n)))
+
+
 def round_bf16(x: float) -> int:
     """bf16 bit pattern of the two-step rounding fp64 -> fp32 -> bf16 (both to nearest even) the RoPE ends with."""
     return int(lib().oracle_round_bf16(float(x)))

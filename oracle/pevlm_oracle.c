@@ -89,6 +89,15 @@ int oracle_num_threads(void) {
 #endif
 }
 
+/* Threads for the following calls from this host thread (a launcher may have pinned OMP_NUM_THREADS to 1). */
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /*
  * Visible key ranges of query row t (Eq. 3-5).  Returns the number of ranges (1 or 2);
  * range r is [lo[r], hi[r]) in global token indices.

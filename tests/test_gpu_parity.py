@@ -372,3 +372,41 @@ def test_bounded_wait_expires_and_the_context_stays_usable():
     ref, lref = oracle.attn_rows(oracle.make_shape(w.S, w.B, w.N, 0, w.Hq, w.Hkv, w.d), qr, kr, v, np.arange(w.L))
     assert np.abs(bits_to_f64(to_bits(o)) - ref).max() <= O_TOL
     assert np.abs(lse.double().cpu().numpy().T - lref).max() <= LSE_TOL
+
+
+# ---------------------------------------------------------------- seeded random shapes (all rows, canary bytes)
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        d = int(rng.choice([64, 128]))
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 3, 4, 7, 8]))
+        S = int(rng.choice([0, int(rng.integers(1, 40)), int(rng.integers(40, 300)), 128, 256]))
+        N = int(rng.integers(0, 5))
+        B = int(rng.choice([int(rng.integers(1, 20)), int(rng.integers(20, 400)), 128, 192])) if N > 0 else 0
+        Q = int(rng.choice([0, 1, int(rng.integers(2, 70))]))
+        if S + N * B + Q == 0:
+            S = 17
+        out.append((S, B, N, Q, Hkv * G, Hkv, d, bool(rng.integers(0, 2)) and S > 0))
+    return out
+
+
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d,outl", _random_shapes(40, seed=20250619))
+def test_random_shapes_match_oracle(S, B, N, Q, Hq, Hkv, d, outl):
+    """Forty seeded shapes drawn over the ranges where the tiling changes form (segments shorter than a tile,
+    ragged tails that are or are not packed across the heads of a group, group sizes 1 to 8, both head
+    dimensions, empty sink / no blocks / no question): every row against the oracle, RoPE and cache bit for bit,
+    canary bytes around every buffer (inside run_gpu_layer)."""
+    w = wl(S, B, N, Q, Hq, Hkv, d, 1e6, outl, seed=4242 + S + 7 * B + 13 * N + Q)
+    q, k, v = inputs.make_qkv(w)
+    res = run_gpu_layer(w, q, k, v)
+    errs, qr, kr = check_against_oracle(w, q, k, v, res, np.arange(w.L))
+    nv = w.n_video
+    np.testing.assert_array_equal(res["q_video"], qr[:nv])
+    np.testing.assert_array_equal(res["q_question"], qr[nv:])
+    np.testing.assert_array_equal(res["k_cache"], kr)
+    np.testing.assert_array_equal(res["v_cache"], v)
+    for name, e in errs.items():
+        assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)

@@ -410,3 +410,27 @@ def test_random_shapes_match_oracle(S, B, N, Q, Hq, Hkv, d, outl):
     np.testing.assert_array_equal(res["v_cache"], v)
     for name, e in errs.items():
         assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)
+
+
+# ---------------------------------------------------------------- the rare in-place rescale of the accumulator
+
+@pytest.mark.parametrize("S,B,N,Q,Hq,Hkv,d", [(300, 400, 2, 40, 8, 2, 128), (140, 520, 1, 9, 4, 2, 64)])
+def test_late_outlier_keys_force_the_accumulator_rescale(S, B, N, Q, Hq, Hkv, d):
+    """The kernel moves a row's reference maximum only when the maximum grows by more than 2^8 and then rescales
+    the row of the output accumulator in place.  With N(0,1) inputs, or outliers among the first sink keys only,
+    that never happens after a row's first key tile.  Here key rows late in the sink, in the middle of the blocks
+    and in the question are scaled by 12 to 40, so the reference maximum jumps in the 2nd, 3rd, ... key tile of
+    rows that follow them (several times for some rows).  Every row against the oracle."""
+    w = wl(S, B, N, Q, Hq, Hkv, d, 1e6, False, seed=31337)
+    late = {S - 7: 12.0, S - 1: 25.0, S + 5: 16.0, S + 131: 30.0, S + B // 2: 20.0, S + B - 2: 40.0}
+    if N > 1:
+        late.update({S + B + 129: 18.0, S + B + 300: 35.0})
+    late.update({w.n_video + Q // 2: 28.0})
+    q = inputs.normal_bf16(w.seed, 1, w.L, Hq, d)
+    k = inputs.normal_bf16(w.seed, 2, w.L, Hkv, d, scale_rows=late)
+    v = inputs.normal_bf16(w.seed, 3, w.L, Hkv, d)
+    res = run_gpu_layer(w, q, k, v)
+    errs, qr, kr = check_against_oracle(w, q, k, v, res, np.arange(w.L))
+    np.testing.assert_array_equal(res["k_cache"], kr)
+    for name, e in errs.items():
+        assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)

@@ -97,6 +97,7 @@ SMALL = [
     (129, 1, 3, 1, 2, 2, 64, 1e4, False),        # blocks of one token
     (257, 384, 2, 130, 8, 2, 128, 1e6, True),    # question longer than a tile's worth of tokens
     (130, 0, 0, 0, 4, 4, 128, 1e6, False),       # sink only
+    (700, 900, 3, 70, 8, 2, 64, 1e6, True),      # head_dim 64 over many tiles: 6 sink + up to 8 block key tiles per item
     (0, 0, 0, 40, 4, 2, 64, 1e4, False),         # question only
 ]
 
@@ -434,3 +435,34 @@ def test_late_outlier_keys_force_the_accumulator_rescale(S, B, N, Q, Hq, Hkv, d)
     np.testing.assert_array_equal(res["k_cache"], kr)
     for name, e in errs.items():
         assert e <= (LSE_TOL if name.startswith("lse") else O_TOL), (name, e, errs)
+
+
+# ---------------------------------------------------------------- RoPE, long-range form of every instantiation
+
+@pytest.mark.parametrize("n,Hq,Hkv,d,sections", [
+    (40000, 2, 1, 64, None),                # plain positions, head_dim 64
+    (10000, 3, 1, 128, (16, 24, 24)),       # multimodal, section boundaries on multiples of 8 pairs
+    (10000, 3, 1, 128, (10, 27, 27)),       # multimodal, a position component per pair
+    (40000, 2, 1, 64, (8, 12, 12)),         # multimodal at head_dim 64
+])
+def test_rope_long_range_forms_bit_exact(n, Hq, Hkv, d, sections):
+    """Token ranges long enough for the RoPE launch to take its long-range form (pairs in shared memory, loads
+    issued ahead), for each instantiation the full-size layer tests do not reach: bit for bit against the oracle."""
+    import torch
+    from paper_2506_19651_b200 import binding as pb
+    w = wl(n, 1, 0, 0, Hq, Hkv, d, 1e6, seed=808)
+    q, k, _ = inputs.make_qkv(w)
+    s = gpu_shape(w)
+    qd, kd = to_dev(q), to_dev(k)
+    qo, ko = torch.empty_like(qd), torch.empty_like(kd)
+    if sections is None:
+        pb.pevlm_rope_qk(s, qd, kd, qo, ko, 1000, n)
+        want_q, want_k = oracle.rope(q, 1e6, first_pos=1000), oracle.rope(k, 1e6, first_pos=1000)
+    else:
+        idx = np.arange(n)
+        pos3 = np.stack([50 + idx // 256, 50 + (idx % 256) // 16, 50 + idx % 16]).astype(np.int32)
+        pb.pevlm_rope_qk_mrope(s, qd, kd, qo, ko, n, torch.from_numpy(pos3).cuda(), sections)
+        want_q, want_k = oracle.rope_mrope(q, 1e6, pos3, sections), oracle.rope_mrope(k, 1e6, pos3, sections)
+    torch.cuda.synchronize()
+    assert_rope_bits(to_bits(qo), want_q, 1)
+    assert_rope_bits(to_bits(ko), want_k, 1)

@@ -98,6 +98,8 @@ SMALL = [
     (257, 384, 2, 130, 8, 2, 128, 1e6, True),    # question longer than a tile's worth of tokens
     (130, 0, 0, 0, 4, 4, 128, 1e6, False),       # sink only
     (700, 900, 3, 70, 8, 2, 64, 1e6, True),      # head_dim 64 over many tiles: 6 sink + up to 8 block key tiles per item
+    (100, 100, 1, 4800, 8, 8, 64, 1e6, True),    # a question block so long that its tiles alone exceed the SM count:
+                                                 # one key split, more work items than CTAs in the question launch
     (0, 0, 0, 40, 4, 2, 64, 1e4, False),         # question only
 ]
 
